@@ -1,0 +1,420 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-KV attention path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One "step" is one pass of the hot path over one batch of the headline workload (a downstream
+operator's suffixes over reused prefix pages): kv_append of the suffix K/V, then attn_extend.
+`value` is the extend algorithmic TFLOP/s over the whole step with inputs resident in HBM; `e2e`
+is the same with host buffers (pinned host -> device copies and the device -> host read of O/LSE
+inside the timed region).  The same line carries the decode (HBM GB/s), bulk-append and mixed
+pipeline-step figures, the roofline of the dominant kernel and the CPU oracle timed on a sample.
+
+Multi-GPU: the path has no exchange step, so N ranks run N independent replicas of the workload
+(different seeds); time is the max over ranks and value the sum of the ranks' work over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2607_23815_b200 import synth  # noqa: E402
+
+METRIC = "paged extend-attn TFLOP/s"
+HEADLINE = "extend_8b"
+
+# DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
+# ncu captures summarised under profiles/; None until a capture of that kernel/workload exists.
+NCU_TRAFFIC_BYTES = {"extend_8b": None, "decode_8b": None}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained"), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def dist_setup(n_gpus):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    return world, rank, local
+
+
+def max_over_ranks(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(x: float, world: int) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device="cuda")
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    torch.cuda.synchronize()
+
+
+class L2Flusher:
+    def __init__(self, device):
+        self.buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)   # 2x the 126 MB L2
+
+    def __call__(self):
+        self.buf.zero_()
+
+
+def time_steps(fn, steps, warmup, flush, world, split=None):
+    """Runs warmup + steps calls of fn(); returns per-step ms (device events) and, if fn records a
+    mid-step event through `split`, the ms of the part after it."""
+    for _ in range(warmup):
+        flush(); fn(None)
+    barrier(world)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
+           torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for i in range(steps):
+        flush()
+        ev[i][0].record()
+        fn(ev[i][1])
+        ev[i][2].record()
+    barrier(world)
+    total = [e[0].elapsed_time(e[2]) for e in ev]
+    tail = [e[1].elapsed_time(e[2]) for e in ev] if split else None
+    return total, tail
+
+
+# --------------------------------------------------------------------------------------------- #
+def cpu_oracle_sample(wl, n_seq, kind):
+    """Times the oracle, as it stands, on the first n_seq sequences of the workload (host cores)."""
+    from oracle import paged_attention as orc
+    g = wl.geom
+    if kind == "extend":
+        s = wl.ext
+        lens = [s.prefix[i] + s.extend[i] for i in range(n_seq)]
+    else:
+        s = wl.dec
+        lens = s.ctx[:n_seq]
+    pages = sum(synth.pages_needed(L, g.page_size) for L in lens)
+    host = orc.PagePool(pages, g.page_size, g.n_kv_heads, g.head_dim)
+    rows, nxt = [], 0
+    for i, L in enumerate(lens):
+        n = synth.pages_needed(L, g.page_size)
+        rows.append(list(range(nxt, nxt + n))); nxt += n
+        kb, vb = wl.gather_host(s.rows[i], L)
+        host.append(rows[-1], 0, kb, vb)
+    bt = synth.block_table(rows)
+    if kind == "extend":
+        E = s.extend[:n_seq]
+        cu = np.concatenate([[0], np.cumsum(E)]).astype(np.int32)
+        qb = synth.bf16_bits(s.q[:int(cu[-1])])
+        t0 = time.perf_counter()
+        o, lse = orc.attn_extend(host, qb, g.n_q_heads, cu, bt, s.prefix[:n_seq], E, g.scale)
+        dt = time.perf_counter() - t0
+        pairs = sum(e * p + e * (e + 1) // 2 for p, e in zip(s.prefix[:n_seq], E))
+        work = 4.0 * g.head_dim * g.n_q_heads * pairs
+        got_o = s.out[:int(cu[-1])].float().cpu().numpy()
+        got_l = s.lse[:int(cu[-1])].cpu().numpy()
+    else:
+        qb = synth.bf16_bits(s.q[:n_seq])
+        t0 = time.perf_counter()
+        o, lse = orc.attn_decode(host, qb, g.n_q_heads, bt, lens, g.scale)
+        dt = time.perf_counter() - t0
+        work = float(sum(lens) * g.kv_bytes_per_token)
+        got_o = s.out[:n_seq].float().cpu().numpy()
+        got_l = s.lse[:n_seq].cpu().numpy()
+    err_o = float(np.max(np.abs(got_o - o)))
+    err_l = float(np.max(np.abs(got_l - lse)))
+    return dt, work, err_o, err_l
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def run_ours(args):
+    world, rank, local = dist_setup(args.gpus)
+    dev = torch.device("cuda", local if world > 1 else 0)
+    torch.cuda.set_device(dev)
+    from paper_2607_23815_b200 import kvattn
+    from paper_2607_23815_b200.workload import DeviceWorkload
+    kvattn.lib()                                                   # fail loudly if the library is missing
+    peaks = load_peaks()
+    flush = L2Flusher(dev)
+    w = synth.WORKLOADS[args.workload]
+    g = w.geom
+    wl = DeviceWorkload(w, dev, seed_offset=rank, write_suffix=True)
+
+    # ---- headline: suffix append + extend attention ----------------------------------------
+    def step(mid_event):
+        wl.append_suffix()
+        if mid_event is not None:
+            mid_event.record()
+        wl.extend()
+
+    sampler = ClockSampler(dev.index or 0) if rank == 0 else None
+    l0 = kvattn.kvattn_launch_count()
+    total_ms, ext_ms = time_steps(step, args.steps, args.warmup, flush, world, split=True)
+    launches = (kvattn.kvattn_launch_count() - l0) * args.steps // (args.steps + args.warmup)
+    clocks = sampler.stop() if sampler else None
+    ms_step = max_over_ranks(statistics.mean(total_ms), world)
+    flops = wl.ext.flops(g)
+    all_flops = sum_over_ranks(flops, world)
+    value = all_flops / (ms_step * 1e-3) / 1e12
+    ext_kernel_ms = statistics.mean(ext_ms)
+    ext_tflops = flops / (ext_kernel_ms * 1e-3) / 1e12
+
+    # ---- e2e: host buffers, copies inside the timed region ---------------------------------
+    e = wl.ext
+    host_in = [t.cpu().pin_memory() for t in (e.q, e.k_new, e.v_new, e.cu_q, e.block_tables, e.prefix_lens, e.extend_lens)]
+    dev_in = [e.q, e.k_new, e.v_new, e.cu_q, e.block_tables, e.prefix_lens, e.extend_lens]
+    host_out = [torch.empty_like(e.out, device="cpu").pin_memory(), torch.empty_like(e.lse, device="cpu").pin_memory()]
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = sum(t.numel() * t.element_size() for t in host_out)
+
+    def e2e_step(_):
+        for h, d in zip(host_in, dev_in):
+            d.copy_(h, non_blocking=True)
+        wl.append_suffix()
+        wl.extend()
+        host_out[0].copy_(e.out, non_blocking=True)
+        host_out[1].copy_(e.lse, non_blocking=True)
+
+    e2e_ms, _ = time_steps(e2e_step, max(3, args.steps // 2), 3, flush, world)
+    e2e_step_ms = max_over_ranks(statistics.mean(e2e_ms), world)
+    e2e_value = all_flops / (e2e_step_ms * 1e-3) / 1e12
+
+    line = {
+        "metric": METRIC, "value": round(value, 3), "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{w.name}: {w.n_extend} tuples, Hq={g.n_q_heads} Hkv={g.n_kv_heads} D={g.head_dim} "
+                               f"page=16, prefix U{list(w.prefix_range)}, extend U{list(w.extend_range)}, "
+                               f"{w.num_pages}-page pool, random placement",
+                   "step": "kv_append(suffix) + attn_extend", "l2": "flushed between steps (256 MiB memset, untimed)",
+                   "multi_gpu": "replicas only (no exchange step)"},
+        "e2e": {"value": round(e2e_value, 3), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": round(e2e_step_ms, 5)},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "tensor", "kernel": "attn_extend", "achieved": round(ext_tflops, 3),
+                     "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(ext_tflops / peaks["bf16_tflops"], 4),
+                     "peak_source": f"{peaks['source']} (burst bf16 matmul)", "frac_of_nominal_2250": round(ext_tflops / 2250.0, 4),
+                     "kernel_ms": round(ext_kernel_ms, 5), "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+        "clocks": clocks,
+    }
+
+    if rank == 0 and world == 1 and not args.headline_only:
+        # ---- CPU oracle on a bounded sample of the same workload ---------------------------
+        n_s = min(args.cpu_sample, len(e.prefix))
+        dt, work, err_o, err_l = cpu_oracle_sample(wl, n_s, "extend")
+        line["cpu_baseline"] = {"value": round(work / dt / 1e12, 6), "unit": "TFLOP/s", "cores": blas_threads(),
+                                "kind": "oracle", "sample": f"first {n_s} of {len(e.prefix)} tuples, {dt:.1f} s",
+                                "max_abs_err_o_vs_gpu": err_o, "max_abs_err_lse_vs_gpu": err_l}
+        wl.close(); del wl
+        torch.cuda.empty_cache()
+        line.update(extra_measurements(args, dev, peaks, flush))
+    else:
+        wl.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+def extra_measurements(args, dev, peaks, flush):
+    """Decode (HBM-bound), bulk append and the mixed pipeline step, each on its own workload."""
+    from paper_2607_23815_b200 import kvattn
+    from paper_2607_23815_b200.workload import DeviceWorkload
+    out = {}
+    steps, warm = max(5, args.steps), 3
+    # decode
+    w = synth.WORKLOADS["decode_8b"]
+    wl = DeviceWorkload(w, dev)
+    ms, _ = time_steps(lambda _: wl.decode(), steps, warm, flush, 1)
+    t = statistics.mean(ms)
+    gbs = wl.dec.kv_bytes(w.geom) / (t * 1e-3) / 1e9
+    dt, work, err_o, err_l = cpu_oracle_sample(wl, min(128, len(wl.dec.ctx)), "decode")
+    out["decode"] = {"workload": f"{w.name}: {w.n_decode} seqs, ctx U{list(w.ctx_range)}, {w.num_pages}-page pool",
+                     "value": round(gbs, 1), "unit": "GB/s", "ms_per_step": round(t, 5), "min_ms": round(min(ms), 5),
+                     "roofline": {"bound": "hbm", "kernel": "attn_decode", "achieved": round(gbs, 1),
+                                  "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
+                                  "peak_source": f"{peaks['source']} (copy)", "frac_of_nominal_8000": round(gbs / 8000.0, 4),
+                                  "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+                     "cpu_baseline": {"value": round(work / dt / 1e9, 4), "unit": "GB/s", "cores": blas_threads(),
+                                      "kind": "oracle", "sample": f"first {min(128, w.n_decode)} of {w.n_decode} sequences, {dt:.1f} s",
+                                      "max_abs_err_o_vs_gpu": err_o, "max_abs_err_lse_vs_gpu": err_l}}
+    # bulk append: re-write every decode sequence's K/V (read + write bytes)
+    d = wl.dec
+    n_tok = sum(d.ctx)
+    if n_tok * w.geom.kv_bytes_per_token < 6 << 30:
+        k_all = torch.empty((n_tok, w.geom.n_kv_heads, w.geom.head_dim), dtype=torch.bfloat16, device=dev).normal_()
+        v_all = torch.empty_like(k_all).normal_()
+        cu = torch.tensor(np.concatenate([[0], np.cumsum(d.ctx)]), dtype=torch.int32, device=dev)
+        zero = torch.zeros(len(d.ctx), dtype=torch.int32, device=dev)
+        ms, _ = time_steps(lambda _: kvattn.kv_append(wl.pool, k_all, v_all, cu, zero, None, d.block_tables),
+                           steps, warm, flush, 1)
+        t = statistics.mean(ms)
+        moved = 2.0 * n_tok * w.geom.kv_bytes_per_token
+        out["append"] = {"workload": f"bulk append of {n_tok} tokens ({moved / 2e9:.2f} GB of K/V)",
+                         "value": round(moved / (t * 1e-3) / 1e9, 1), "unit": "GB/s (read+write)",
+                         "ms_per_step": round(t, 5),
+                         "frac_of_measured_copy": round(moved / (t * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+        del k_all, v_all
+    wl.close(); del wl
+    torch.cuda.empty_cache()
+    # mixed pipeline step
+    w = synth.WORKLOADS["pipeline_step"]
+    wl = DeviceWorkload(w, dev)
+    ms_mixed, _ = time_steps(lambda _: wl.mixed(), steps, warm, flush, 1)
+    ms_ext, _ = time_steps(lambda _: wl.extend(), steps, warm, flush, 1)
+    ms_dec, _ = time_steps(lambda _: wl.decode(), steps, warm, flush, 1)
+    out["pipeline_step"] = {"workload": f"{w.name}: {w.n_extend} extend + {w.n_decode} decode sequences",
+                            "mixed_ms": round(statistics.mean(ms_mixed), 5),
+                            "extend_alone_ms": round(statistics.mean(ms_ext), 5),
+                            "decode_alone_ms": round(statistics.mean(ms_dec), 5),
+                            "extend_tflops_alone": round(wl.ext.flops(w.geom) / statistics.mean(ms_ext) / 1e9, 2),
+                            "decode_gbs_alone": round(wl.dec.kv_bytes(w.geom) / statistics.mean(ms_dec) / 1e6, 1)}
+    wl.close()
+    return out
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import paged_attention as orc
+    w = synth.WORKLOADS[args.workload]
+    g = w.geom
+    ext, _ = synth.draw_lengths(w)
+    n_s = min(args.cpu_sample, len(ext))
+    P, E = [p for p, _ in ext[:n_s]], [e for _, e in ext[:n_s]]
+    pages = sum(synth.pages_needed(p + e, g.page_size) for p, e in zip(P, E))
+    host = orc.PagePool(pages, g.page_size, g.n_kv_heads, g.head_dim)
+    perm = synth.page_permutation(w.seed, pages).tolist()
+    rows, qs = [], []
+    for i in range(n_s):
+        L = P[i] + E[i]
+        n = synth.pages_needed(L, g.page_size)
+        rows.append(perm[:n]); perm = perm[n:]
+        host.append(rows[-1], 0,
+                    synth.bf16_bits(synth.normal_bf16(w.seed, synth.TAG_K, i, 0, L, g.n_kv_heads, g.head_dim)),
+                    synth.bf16_bits(synth.normal_bf16(w.seed, synth.TAG_V, i, 0, L, g.n_kv_heads, g.head_dim)))
+        qs.append(synth.bf16_bits(synth.normal_bf16(w.seed, synth.TAG_Q, i, P[i], E[i], g.n_q_heads, g.head_dim)))
+    q = np.concatenate(qs)
+    cu = np.concatenate([[0], np.cumsum(E)]).astype(np.int32)
+    bt = synth.block_table(rows)
+    flops = 4.0 * g.head_dim * g.n_q_heads * sum(e * p + e * (e + 1) // 2 for p, e in zip(P, E))
+    times = []
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        orc.attn_extend(host, q, g.n_q_heads, cu, bt, P, E, g.scale)
+        if i >= args.warmup:
+            times.append(time.perf_counter() - t0)
+    t = statistics.mean(times)
+    v = round(flops / t / 1e12, 6)
+    sample = f"first {n_s} of {len(ext)} tuples per step (gather + attention, K/V already in host pages)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(t * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name} (sample)", "sample": sample},
+        "cpu_baseline": {"value": v, "unit": "TFLOP/s", "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=HEADLINE, choices=[k for k, v in synth.WORKLOADS.items() if v.n_extend])
+    ap.add_argument("--cpu-sample", type=int, default=64, help="tuples in the CPU-oracle sample")
+    ap.add_argument("--headline-only", action="store_true", help="skip the decode/append/mixed extras")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,189 @@
+/*
+ * kvattn.h - C ABI of a B200 (sm_100a) library for attention over a paged KV-cache pool.
+ *
+ * The calls follow the problem as the paper states it (arxiv 2607.23815, "Kalypso:
+ * Relational LLM Serving"): an inference engine keeps K/V tensors in a global pool of
+ * fixed-size blocks (pages) that are handed out when a request is admitted and returned
+ * when it completes (Section 2.1, "vLLM memory model"); when a downstream semantic
+ * operator's prompt shares its prefix with the upstream operator's prompt for the same
+ * tuple, the cached KV entries are reused and only the new suffix is prefilled
+ * (Section 2.1, "Prefix caching" and "Prefix sharing in semantic operators"); short
+ * answers are then decoded one token at a time over all stored K/V (Section 2.1, first
+ * paragraph); the scheduler releases a task's memory when the tuple is filtered or has
+ * left the last stage (Algorithm 1, Complete), and unpinned blocks may be evicted under
+ * memory pressure (Section 2.1; Section 6, "Explicit and virtual pinning").
+ *
+ * Conventions that hold for every call
+ *  - Pointers are marked [host] or [dev].  The library never keeps a caller pointer past
+ *    the call, and never frees or reallocates caller memory.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Calls
+ *    that take a stream enqueue work and return without synchronising.
+ *  - Every call returns a kv_status_t.  Errors that the host can see (NULL pointers,
+ *    negative sizes, unsupported shapes, a workspace that is too small) are returned at
+ *    once with nothing launched.  Problems only the device can see (a block-table entry
+ *    outside the pool) make the kernel skip the access and record KV_ERR_BOUNDS in a
+ *    device status word that kv_last_async_status() reads.  Nothing aborts, traps or throws.
+ *  - Supported shapes: bf16 K/V/Q/O, page_size 16, head_dim 64 or 128,
+ *    group G = n_q_heads / n_kv_heads in {1, 2, 4, 8}.  Anything else: KV_ERR_UNSUPPORTED.
+ *  - All integer arrays are int32.  Block tables are row-major [rows][max_pages]; entry b
+ *    of a row is the physical page of logical block b (tokens 16b .. 16b+15); entries past
+ *    ceil(len/16) are never read (pad with -1).
+ *
+ * Page layout in device memory (private to the library, documented for tests)
+ *    K and V are two buffers of num_pages * n_kv_heads blocks; block (page, head) holds the
+ *    16 tokens x head_dim bf16 values of that page and KV head, contiguous, 16*head_dim*2
+ *    bytes.  Inside a block, element (slot, d) lives at byte offset
+ *        (slot/8) * (8*head_dim*2) + (d/64) * 1024 + (slot%8) * 128
+ *            + ((((d%64)/8) ^ (slot%8)) * 16) + (d%8) * 2
+ *    i.e. 8-token x 64-dim tiles of 1024 bytes whose 16-byte chunks are XOR-swizzled by the
+ *    row index.  This is the 128-byte-swizzle shared-memory operand layout of the sm_100
+ *    tensor-core MMA, so one bulk copy brings a block into shared memory ready for use.
+ *    kv_pool_elem_offset() evaluates the formula.
+ */
+#ifndef KVATTN_H_
+#define KVATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kv_pool kv_pool_t; /* opaque: owns the K/V page memory and the host free list */
+
+typedef enum {
+  KV_OK = 0,
+  KV_ERR_INVALID = 1,       /* NULL pointer, negative size, inconsistent arguments            */
+  KV_ERR_OOM = 2,           /* kv_alloc: not enough free pages (the caller defers the request) */
+  KV_ERR_NOT_ALLOCATED = 3, /* kv_free / kv_evict of a page that is not allocated               */
+  KV_ERR_BOUNDS = 4,        /* device saw a block-table entry or length outside the pool      */
+  KV_ERR_UNSUPPORTED = 5,   /* shape outside the supported set                                 */
+  KV_ERR_CUDA = 6,          /* a CUDA runtime call failed (allocation, launch)                 */
+  KV_ERR_TIMEOUT = 7,       /* a bounded device-side wait gave up                              */
+  KV_ERR_WORKSPACE = 8      /* workspace pointer NULL or smaller than attn_workspace_bytes()   */
+} kv_status_t;
+
+const char* kv_status_str(kv_status_t s);
+
+/* ---- pool: "a global pool of fixed-size blocks" (Section 2.1, vLLM memory model) ---------- */
+
+/* Creates a pool on the current CUDA device and allocates its K and V buffers with cudaMalloc
+ * (2 * num_pages * n_kv_heads * page_size * head_dim * 2 bytes).  *out receives the handle. */
+kv_status_t kv_pool_create(int num_pages, int page_size, int n_kv_heads, int head_dim, kv_pool_t** out);
+/* Same, over caller-owned device buffers k_base/v_base [dev] of at least that size each, 256-byte
+ * aligned; the pool does not free them.  Lets a framework place the pages in its own allocator. */
+kv_status_t kv_pool_create_ex(int num_pages, int page_size, int n_kv_heads, int head_dim, void* k_base,
+                              void* v_base, kv_pool_t** out);
+/* Frees what the pool owns.  The caller makes sure no kernel using the pool is still running. */
+kv_status_t kv_pool_destroy(kv_pool_t* pool);
+/* Occupancy as the scheduler reads it from the engine (Section 3): any pointer may be NULL. */
+kv_status_t kv_pool_stats(const kv_pool_t* pool, int* free_pages, int* used_pages, int64_t* evicted_total);
+/* Test surface: device base pointers and the size in bytes of each of the two buffers. */
+kv_status_t kv_pool_raw(const kv_pool_t* pool, void** k_base, void** v_base, int64_t* bytes_each);
+/* Test surface: ELEMENT offset (bf16 units) of (page, kv_head, slot, d) from k_base / v_base per
+ * the layout formula above; -1 if out of range. */
+int64_t kv_pool_elem_offset(const kv_pool_t* pool, int page, int kv_head, int slot, int d);
+/* Debug aid: when on, kv_evict() overwrites the evicted pages with NaN bit patterns (on the legacy
+ * default stream, synchronously) so that a stale read shows up in outputs. */
+kv_status_t kv_pool_set_poison(kv_pool_t* pool, int on);
+
+/* ---- allocator (host; mutex-guarded) ------------------------------------------------------ */
+
+/* Hands out n page ids into out_page_ids [host].  All-or-nothing: KV_ERR_OOM leaves the pool
+ * unchanged ("if insufficient blocks are available, new requests are deferred", Section 2.1).
+ * Order is deterministic: a fresh pool gives 0,1,2,...; released pages come back last-in-first-out. */
+kv_status_t kv_alloc(kv_pool_t* pool, int n, int* out_page_ids);
+/* Returns pages whose owner is done (Algorithm 1, Complete: releaseMemory).  A page id that is out
+ * of range, not allocated, or listed twice gives KV_ERR_NOT_ALLOCATED with no partial effect. */
+kv_status_t kv_free(kv_pool_t* pool, const int* page_ids /*host*/, int n);
+/* Returns pages reclaimed under memory pressure (Section 2.1: completed requests' blocks "may be
+ * evicted at any time").  Same as kv_free plus the eviction counter and the optional poison fill;
+ * the former owner must treat its prefix as lost and re-prefill (Section 2.2). */
+kv_status_t kv_evict(kv_pool_t* pool, const int* page_ids /*host*/, int n);
+
+/* ---- kv_append: materialise new tokens' K/V in their pages (Section 2.1: prefill "materializes
+ *      per-layer key-value tensors") ------------------------------------------------------- */
+/* n_segments segments; segment s holds rows cu_new[s] .. cu_new[s+1]-1 of k_new/v_new
+ * ([dev] bf16 [total_new][n_kv_heads][head_dim]) and writes them to token positions
+ * start_pos[s] .. of the sequence whose block-table row is seg_row[s] (seg_row NULL: row s).
+ * cu_new [dev][n_segments+1], start_pos [dev][n_segments], seg_row [dev][n_segments] or NULL,
+ * block_tables [dev][rows][max_pages].  Segments must not overlap each other.  Pure data movement:
+ * the stored bits equal the input bits. */
+kv_status_t kv_append(kv_pool_t* pool, const void* k_new, const void* v_new, const int* cu_new,
+                      const int* start_pos, const int* seg_row, const int* block_tables, int max_pages,
+                      int n_segments, int total_new, void* stream);
+
+/* Debug/test surface: copies tokens 0..len-1 of one sequence out of its pages into contiguous
+ * k_out/v_out [dev] bf16 [len][n_kv_heads][head_dim].  block_table_row [dev][>= ceil(len/16)]. */
+kv_status_t kv_gather(kv_pool_t* pool, const int* block_table_row, int len, void* k_out, void* v_out,
+                      void* stream);
+
+/* ---- attention ---------------------------------------------------------------------------- */
+/* Common definition (Section 2.1; the plain softmax attention the engine computes): for a query
+ * row q of head h at absolute position p, with KV head g = h / G,
+ *     s_j = scale * <q, k_j>,  j = 0..p;   O = sum_j softmax(s)_j v_j;   LSE = ln sum_j exp(s_j).
+ * O is written as bf16 (fp32 accumulation, one rounding at the store), LSE as fp32 (natural log). */
+
+/* Bytes of scratch [dev] the attention calls need for the given batch (256-byte aligned). */
+size_t attn_workspace_bytes(const kv_pool_t* pool, int n_q_heads, int batch_ext, int total_q, int max_total_len,
+                            int batch_dec, int max_ctx_len);
+
+/* Extend ("only prefills the ... suffix", Section 2.1): sequence i has prefix_lens[i] reused tokens
+ * and extend_lens[i] new ones, all already in its pages (kv_append first).  Suffix token t sits at
+ * position prefix_lens[i]+t and sees keys 0..prefix_lens[i]+t.  prefix_lens[i]=0 is a from-scratch
+ * prefill (the cache-miss path of Section 2.2); extend_lens[i]=0 contributes no rows.
+ * q/out [dev] bf16 [total_q][n_q_heads][head_dim], ragged by cu_q [dev][batch+1]; lse [dev] fp32
+ * [total_q][n_q_heads]; prefix_lens, extend_lens [dev][batch].  max_extend_len / max_total_len are
+ * host-side upper bounds on extend_lens[i] and prefix_lens[i]+extend_lens[i] (they size the grid). */
+kv_status_t attn_extend(kv_pool_t* pool, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                        int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                        int max_extend_len, int max_total_len, float scale, void* out, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+/* Decode ("one token at a time, attending over all previously computed KV", Section 2.1): one query
+ * per sequence at position ctx_lens[i]-1 over keys 0..ctx_lens[i]-1 (its own K/V already appended).
+ * q/out [dev] bf16 [batch][n_q_heads][head_dim]; lse [dev] fp32 [batch][n_q_heads]; ctx_lens [dev]
+ * [batch]; max_ctx_len: host upper bound.  ctx_lens[i] <= 0 writes O = 0, LSE = -inf. */
+kv_status_t attn_decode(kv_pool_t* pool, const void* q, int n_q_heads, const int* block_tables, int max_pages,
+                        const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream);
+
+typedef struct {
+  const void* q; const int* cu_q; const int* block_tables; int max_pages;
+  const int* prefix_lens; const int* extend_lens; int batch; int total_q;
+  int max_extend_len; int max_total_len; void* out; float* lse;
+} attn_extend_args_t;
+
+typedef struct {
+  const void* q; const int* block_tables; int max_pages; const int* ctx_lens;
+  int batch; int max_ctx_len; void* out; float* lse;
+} attn_decode_args_t;
+
+/* One pipeline step of two chained operators (e.g. sem_map feeding sem_filter, Section 1): the
+ * extend set and the decode set are launched so that the tensor-bound and the HBM-bound work
+ * share the GPU.  Either argument may be NULL or have batch 0.  The workspace must be sized by
+ * attn_workspace_bytes() with both batches.  Work is ordered after prior work on `stream`, and
+ * later work on `stream` is ordered after it. */
+kv_status_t attn_mixed(kv_pool_t* pool, int n_q_heads, float scale, const attn_extend_args_t* ext,
+                       const attn_decode_args_t* dec, void* workspace, size_t workspace_bytes, void* stream);
+
+/* ---- checks ------------------------------------------------------------------------------- */
+/* Validates on the device that every block-table entry a batch would read (blocks 0..ceil(len/16)-1
+ * of each row) is a page of this pool and that 0 <= lens[i] <= 16*max_pages; synchronises; returns
+ * KV_ERR_BOUNDS if not.  lens, block_tables [dev]. */
+kv_status_t kv_check_batch(kv_pool_t* pool, const int* block_tables, int max_pages, const int* lens, int batch,
+                           void* stream);
+/* Synchronises the device, returns and clears the device status word (KV_OK if nothing was seen). */
+kv_status_t kv_last_async_status(kv_pool_t* pool);
+
+/* Selects the extend kernel: 0 = automatic, 1 = the small-tile kernel (rows of one KV head read K/V
+ * straight from HBM), 2 = the tcgen05 tensor-core kernel.  Process-wide; for tests and benchmarks. */
+kv_status_t kvattn_set_extend_impl(int impl);
+/* Number of kernels this library has launched since load (all pools); for benchmark accounting. */
+int64_t kvattn_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVATTN_H_ */

@@ -1,0 +1,130 @@
+// Public attention entry points: argument checks, kernel selection, the mixed-batch launcher.
+#include "common.cuh"
+
+namespace kvattn {
+size_t decode_workspace_bytes(int n_q_heads, int head_dim, int batch, int max_ctx_len);
+kv_status_t launch_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
+                          const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
+                          void* workspace, size_t workspace_bytes, cudaStream_t st);
+kv_status_t launch_extend_small(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                                int max_pages, const int* prefix_lens, const int* extend_lens, int batch,
+                                int max_extend_len, int max_total_len, float scale, void* out, float* lse,
+                                cudaStream_t st);
+size_t extend_tc_workspace_bytes(int n_q_heads, int head_dim, int batch, int total_q, int max_total_len);
+bool extend_tc_supported(const kv_pool_t* p, int n_q_heads);
+kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                             int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                             int max_extend_len, int max_total_len, float scale, void* out, float* lse,
+                             void* workspace, size_t workspace_bytes, cudaStream_t st);
+
+static std::atomic<int> g_extend_impl{0};
+
+static bool heads_supported(const kv_pool_t* p, int n_q_heads) {
+  if (n_q_heads <= 0 || n_q_heads % p->n_kv_heads != 0) return false;
+  const int g = n_q_heads / p->n_kv_heads;
+  return g == 1 || g == 2 || g == 4 || g == 8;
+}
+
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+}  // namespace kvattn
+
+using namespace kvattn;
+
+extern "C" {
+
+kv_status_t kvattn_set_extend_impl(int impl) {
+  if (impl < 0 || impl > 2) return KV_ERR_INVALID;
+  g_extend_impl.store(impl);
+  return KV_OK;
+}
+
+size_t attn_workspace_bytes(const kv_pool_t* p, int n_q_heads, int batch_ext, int total_q, int max_total_len,
+                            int batch_dec, int max_ctx_len) {
+  if (p == nullptr || n_q_heads <= 0) return 0;
+  // the two regions are disjoint so that a mixed step can run both kinds of work at once
+  return align256(extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch_ext, total_q, max_total_len)) +
+         align256(decode_workspace_bytes(n_q_heads, p->head_dim, batch_dec, max_ctx_len)) + 256;
+}
+
+kv_status_t attn_extend(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                        int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                        int max_extend_len, int max_total_len, float scale, void* out, float* lse, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+  if (p == nullptr || batch < 0 || total_q < 0 || max_pages < 0 || max_extend_len < 0 || max_total_len < 0)
+    return KV_ERR_INVALID;
+  if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
+  if (batch == 0 || total_q == 0 || max_extend_len == 0) return KV_OK;
+  if (q == nullptr || cu_q == nullptr || block_tables == nullptr || prefix_lens == nullptr ||
+      extend_lens == nullptr || out == nullptr || lse == nullptr)
+    return KV_ERR_INVALID;
+  if ((((uintptr_t)q) | ((uintptr_t)out)) & 15) return KV_ERR_INVALID;
+  if (max_total_len < max_extend_len || max_total_len > (int64_t)max_pages * kPageSize) return KV_ERR_INVALID;
+  const int impl = g_extend_impl.load();
+  const bool tc_ok = extend_tc_supported(p, n_q_heads);
+  if (impl == 2 && !tc_ok) return KV_ERR_UNSUPPORTED;
+  if (impl == 2 || (impl == 0 && tc_ok)) {
+    return launch_extend_tc(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
+                            max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes,
+                            (cudaStream_t)stream);
+  }
+  return launch_extend_small(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch,
+                             max_extend_len, max_total_len, scale, out, lse, (cudaStream_t)stream);
+}
+
+kv_status_t attn_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
+                        const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  if (p == nullptr || batch < 0 || max_pages < 0 || max_ctx_len < 0) return KV_ERR_INVALID;
+  if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
+  if (batch == 0) return KV_OK;
+  if (q == nullptr || block_tables == nullptr || ctx_lens == nullptr || out == nullptr || lse == nullptr)
+    return KV_ERR_INVALID;
+  if ((((uintptr_t)q) | ((uintptr_t)out)) & 15) return KV_ERR_INVALID;
+  if (max_ctx_len > (int64_t)max_pages * kPageSize) return KV_ERR_INVALID;
+  if (max_ctx_len == 0) max_ctx_len = 1;  // every row is empty: still defines O = 0, LSE = -inf
+  // the decode region of a combined workspace starts after the extend region; a caller that sized
+  // the workspace for decode only passes (0, 0) for the extend part, so the offset is 0 there
+  return launch_decode(p, q, n_q_heads, block_tables, max_pages, ctx_lens, batch, max_ctx_len, scale, out, lse,
+                       workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+kv_status_t attn_mixed(kv_pool_t* p, int n_q_heads, float scale, const attn_extend_args_t* ext,
+                       const attn_decode_args_t* dec, void* workspace, size_t workspace_bytes, void* stream) {
+  if (p == nullptr) return KV_ERR_INVALID;
+  if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
+  const bool has_ext = ext != nullptr && ext->batch > 0 && ext->total_q > 0;
+  const bool has_dec = dec != nullptr && dec->batch > 0;
+  cudaStream_t st = (cudaStream_t)stream;
+  size_t ext_bytes = 0;
+  if (has_ext)
+    ext_bytes = align256(extend_tc_workspace_bytes(n_q_heads, p->head_dim, ext->batch, ext->total_q, ext->max_total_len));
+  if (ext_bytes > workspace_bytes) return KV_ERR_WORKSPACE;
+  char* ws = reinterpret_cast<char*>(workspace);
+  if (has_ext && has_dec) {
+    // decode (HBM-bound) goes to the pool's side stream, extend (tensor-bound) stays on the caller's
+    KV_CUDA_OK(cudaEventRecord(p->ev_fork, st));
+    KV_CUDA_OK(cudaStreamWaitEvent(p->side_stream, p->ev_fork, 0));
+    kv_status_t s = attn_decode(p, dec->q, n_q_heads, dec->block_tables, dec->max_pages, dec->ctx_lens, dec->batch,
+                                dec->max_ctx_len, scale, dec->out, dec->lse, ws ? ws + ext_bytes : nullptr,
+                                workspace_bytes - ext_bytes, p->side_stream);
+    kv_status_t s2 = KV_OK;
+    if (s == KV_OK)
+      s2 = attn_extend(p, ext->q, n_q_heads, ext->cu_q, ext->block_tables, ext->max_pages, ext->prefix_lens,
+                       ext->extend_lens, ext->batch, ext->total_q, ext->max_extend_len, ext->max_total_len, scale,
+                       ext->out, ext->lse, ws, ext_bytes, st);
+    // always rejoin, so that the caller's stream stays ordered after whatever was launched
+    KV_CUDA_OK(cudaEventRecord(p->ev_join, p->side_stream));
+    KV_CUDA_OK(cudaStreamWaitEvent(st, p->ev_join, 0));
+    return s != KV_OK ? s : s2;
+  }
+  if (has_ext)
+    return attn_extend(p, ext->q, n_q_heads, ext->cu_q, ext->block_tables, ext->max_pages, ext->prefix_lens,
+                       ext->extend_lens, ext->batch, ext->total_q, ext->max_extend_len, ext->max_total_len, scale,
+                       ext->out, ext->lse, ws, ext_bytes, st);
+  if (has_dec)
+    return attn_decode(p, dec->q, n_q_heads, dec->block_tables, dec->max_pages, dec->ctx_lens, dec->batch,
+                       dec->max_ctx_len, scale, dec->out, dec->lse, ws, workspace_bytes, st);
+  return KV_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,334 @@
+// Page pool, allocator and the data-movement kernels (append, gather, bounds check, poison).
+#include <algorithm>
+#include <new>
+
+#include "common.cuh"
+
+namespace kvattn {
+
+std::atomic<int64_t> g_launches{0};
+
+// ------------------------------------------------------------------------------------------
+// kv_append: one thread moves one 16-byte chunk of K and the matching chunk of V.
+// Consecutive threads read consecutive chunks of a token row (coalesced 16-byte loads); the
+// eight chunks of a 64-dim half land, permuted, in one 128-byte row of the page (full-line
+// 16-byte stores).
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) append_kernel(PoolView pool, const uint4* __restrict__ k_new,
+                                                     const uint4* __restrict__ v_new,
+                                                     const int* __restrict__ cu_new,
+                                                     const int* __restrict__ start_pos,
+                                                     const int* __restrict__ seg_row,
+                                                     const int* __restrict__ block_tables, int max_pages,
+                                                     int n_segments, int total_new) {
+  const int chunks_per_row = pool.head_dim >> 3;               // 16-byte chunks per (token, head)
+  const int chunks_per_token = pool.n_kv_heads * chunks_per_row;
+  const int64_t total = (int64_t)total_new * chunks_per_token;
+  const size_t blk = block_bytes(pool.head_dim);
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int token = (int)(idx / chunks_per_token);
+    const int rem = (int)(idx - (int64_t)token * chunks_per_token);
+    const int head = rem / chunks_per_row;
+    const int dchunk = rem - head * chunks_per_row;
+    // segment of this token: last s with cu_new[s] <= token
+    int lo = 0, hi = n_segments;
+    while (hi - lo > 1) {
+      const int mid = (lo + hi) >> 1;
+      if (__ldg(cu_new + mid) <= token) lo = mid; else hi = mid;
+    }
+    const int seg = lo;
+    const int seg_begin = __ldg(cu_new + seg);
+    if (token >= __ldg(cu_new + seg + 1)) continue;            // cu_new not covering this row: skip
+    const int pos = __ldg(start_pos + seg) + (token - seg_begin);
+    const int row = seg_row ? __ldg(seg_row + seg) : seg;
+    const int blk_idx = pos >> 4;
+    if (pos < 0 || blk_idx >= max_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
+    const int page = __ldg(block_tables + (int64_t)row * max_pages + blk_idx);
+    if (page < 0 || page >= pool.num_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
+    const size_t off = ((size_t)page * pool.n_kv_heads + head) * blk + chunk_offset_bytes(pos & 15, dchunk, pool.head_dim);
+    const uint4 kk = __ldg(k_new + idx);
+    const uint4 vv = __ldg(v_new + idx);
+    *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + off) = kk;
+    *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + off) = vv;
+  }
+}
+
+__global__ void __launch_bounds__(256) gather_kernel(PoolView pool, const int* __restrict__ block_row, int len,
+                                                     uint4* __restrict__ k_out, uint4* __restrict__ v_out) {
+  const int chunks_per_row = pool.head_dim >> 3;
+  const int chunks_per_token = pool.n_kv_heads * chunks_per_row;
+  const int64_t total = (int64_t)len * chunks_per_token;
+  const size_t blk = block_bytes(pool.head_dim);
+  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+       idx += (int64_t)gridDim.x * blockDim.x) {
+    const int token = (int)(idx / chunks_per_token);
+    const int rem = (int)(idx - (int64_t)token * chunks_per_token);
+    const int head = rem / chunks_per_row;
+    const int dchunk = rem - head * chunks_per_row;
+    const int page = __ldg(block_row + (token >> 4));
+    if (page < 0 || page >= pool.num_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
+    const size_t off = ((size_t)page * pool.n_kv_heads + head) * blk + chunk_offset_bytes(token & 15, dchunk, pool.head_dim);
+    k_out[idx] = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(pool.k) + off);
+    v_out[idx] = *reinterpret_cast<const uint4*>(reinterpret_cast<const char*>(pool.v) + off);
+  }
+}
+
+__global__ void check_batch_kernel(PoolView pool, const int* __restrict__ block_tables, int max_pages,
+                                   const int* __restrict__ lens, int batch) {
+  for (int i = blockIdx.x; i < batch; i += gridDim.x) {
+    const int len = lens[i];
+    if (len < 0 || len > max_pages * kPageSize) {
+      if (threadIdx.x == 0) report(pool.status, KV_ERR_BOUNDS);
+      continue;
+    }
+    const int nblk = (len + kPageSize - 1) / kPageSize;
+    for (int b = threadIdx.x; b < nblk; b += blockDim.x) {
+      const int page = block_tables[(int64_t)i * max_pages + b];
+      if (page < 0 || page >= pool.num_pages) report(pool.status, KV_ERR_BOUNDS);
+    }
+  }
+}
+
+__global__ void poison_kernel(PoolView pool, const int* __restrict__ page_ids, int n) {
+  const size_t per_page16 = (block_bytes(pool.head_dim) * pool.n_kv_heads) >> 4;
+  const uint4 nan4 = make_uint4(0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu);
+  for (int i = blockIdx.x; i < n; i += gridDim.x) {
+    const int page = page_ids[i];
+    if (page < 0 || page >= pool.num_pages) continue;
+    uint4* kp = reinterpret_cast<uint4*>(pool.k) + (size_t)page * per_page16;
+    uint4* vp = reinterpret_cast<uint4*>(pool.v) + (size_t)page * per_page16;
+    for (size_t j = threadIdx.x; j < per_page16; j += blockDim.x) { kp[j] = nan4; vp[j] = nan4; }
+  }
+}
+
+static bool shape_supported(int page_size, int n_kv_heads, int head_dim) {
+  return page_size == kPageSize && (head_dim == 64 || head_dim == 128) && n_kv_heads >= 1;
+}
+
+static int grid_for(int64_t work_items, int threads) {
+  int64_t blocks = (work_items + threads - 1) / threads;
+  const int64_t cap = 148 * 16;  // a few waves of resident blocks; grid-stride covers the rest
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  return (int)blocks;
+}
+
+}  // namespace kvattn
+
+using namespace kvattn;
+
+extern "C" {
+
+const char* kv_status_str(kv_status_t s) {
+  switch (s) {
+    case KV_OK: return "ok";
+    case KV_ERR_INVALID: return "invalid argument";
+    case KV_ERR_OOM: return "out of pages";
+    case KV_ERR_NOT_ALLOCATED: return "page not allocated";
+    case KV_ERR_BOUNDS: return "block table entry or length out of bounds";
+    case KV_ERR_UNSUPPORTED: return "unsupported shape";
+    case KV_ERR_CUDA: return "CUDA runtime error";
+    case KV_ERR_TIMEOUT: return "device-side wait timed out";
+    case KV_ERR_WORKSPACE: return "workspace missing or too small";
+  }
+  return "unknown status";
+}
+
+static kv_status_t pool_create_impl(int num_pages, int page_size, int n_kv_heads, int head_dim, void* k_base,
+                                    void* v_base, bool owns, kv_pool_t** out) {
+  if (out == nullptr) return KV_ERR_INVALID;
+  *out = nullptr;
+  if (num_pages <= 0 || n_kv_heads <= 0) return KV_ERR_INVALID;
+  if (!shape_supported(page_size, n_kv_heads, head_dim)) return KV_ERR_UNSUPPORTED;
+  kv_pool* p = new (std::nothrow) kv_pool();
+  if (p == nullptr) return KV_ERR_OOM;
+  p->num_pages = num_pages; p->page_size = page_size; p->n_kv_heads = n_kv_heads; p->head_dim = head_dim;
+  p->owns_buffers = owns; p->k_base = k_base; p->v_base = v_base;
+  p->bytes_each = (int64_t)num_pages * n_kv_heads * (int64_t)block_bytes(head_dim);
+  p->d_status = nullptr; p->d_scratch_ids = nullptr; p->poison = false;
+  p->side_stream = nullptr; p->ev_fork = nullptr; p->ev_join = nullptr;
+  p->mark_epoch = 0; p->evicted_total = 0;
+  bool ok = cudaGetDevice(&p->device) == cudaSuccess;
+  if (ok && owns) {
+    ok = cudaMalloc(&p->k_base, (size_t)p->bytes_each) == cudaSuccess &&
+         cudaMalloc(&p->v_base, (size_t)p->bytes_each) == cudaSuccess;
+  }
+  ok = ok && cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess &&
+       cudaMemset(p->d_status, 0, sizeof(int)) == cudaSuccess &&
+       cudaMalloc(&p->d_scratch_ids, sizeof(int) * (size_t)num_pages) == cudaSuccess &&
+       cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking) == cudaSuccess &&
+       cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
+       cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) {
+    kv_pool_destroy(p);
+    cudaGetLastError();
+    return KV_ERR_CUDA;
+  }
+  p->free_stack.resize(num_pages);
+  for (int i = 0; i < num_pages; ++i) p->free_stack[i] = num_pages - 1 - i;  // back() == 0 first
+  p->allocated.assign(num_pages, 0);
+  p->mark.assign(num_pages, 0);
+  *out = p;
+  return KV_OK;
+}
+
+kv_status_t kv_pool_create(int num_pages, int page_size, int n_kv_heads, int head_dim, kv_pool_t** out) {
+  return pool_create_impl(num_pages, page_size, n_kv_heads, head_dim, nullptr, nullptr, true, out);
+}
+
+kv_status_t kv_pool_create_ex(int num_pages, int page_size, int n_kv_heads, int head_dim, void* k_base,
+                              void* v_base, kv_pool_t** out) {
+  if (k_base == nullptr || v_base == nullptr) return KV_ERR_INVALID;
+  if (((uintptr_t)k_base & 255) != 0 || ((uintptr_t)v_base & 255) != 0) return KV_ERR_INVALID;
+  return pool_create_impl(num_pages, page_size, n_kv_heads, head_dim, k_base, v_base, false, out);
+}
+
+kv_status_t kv_pool_destroy(kv_pool_t* p) {
+  if (p == nullptr) return KV_ERR_INVALID;
+  if (p->owns_buffers) {
+    if (p->k_base) cudaFree(p->k_base);
+    if (p->v_base) cudaFree(p->v_base);
+  }
+  if (p->d_status) cudaFree(p->d_status);
+  if (p->d_scratch_ids) cudaFree(p->d_scratch_ids);
+  if (p->side_stream) cudaStreamDestroy(p->side_stream);
+  if (p->ev_fork) cudaEventDestroy(p->ev_fork);
+  if (p->ev_join) cudaEventDestroy(p->ev_join);
+  delete p;
+  return KV_OK;
+}
+
+kv_status_t kv_pool_stats(const kv_pool_t* p, int* free_pages, int* used_pages, int64_t* evicted_total) {
+  if (p == nullptr) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(const_cast<kv_pool_t*>(p)->mu);
+  if (free_pages) *free_pages = (int)p->free_stack.size();
+  if (used_pages) *used_pages = p->num_pages - (int)p->free_stack.size();
+  if (evicted_total) *evicted_total = p->evicted_total;
+  return KV_OK;
+}
+
+kv_status_t kv_pool_raw(const kv_pool_t* p, void** k_base, void** v_base, int64_t* bytes_each) {
+  if (p == nullptr) return KV_ERR_INVALID;
+  if (k_base) *k_base = p->k_base;
+  if (v_base) *v_base = p->v_base;
+  if (bytes_each) *bytes_each = p->bytes_each;
+  return KV_OK;
+}
+
+int64_t kv_pool_elem_offset(const kv_pool_t* p, int page, int kv_head, int slot, int d) {
+  if (p == nullptr || page < 0 || page >= p->num_pages || kv_head < 0 || kv_head >= p->n_kv_heads || slot < 0 ||
+      slot >= p->page_size || d < 0 || d >= p->head_dim)
+    return -1;
+  const int64_t blk_elems = (int64_t)p->page_size * p->head_dim;
+  return ((int64_t)page * p->n_kv_heads + kv_head) * blk_elems +
+         (int64_t)(chunk_offset_bytes(slot, d >> 3, p->head_dim) >> 1) + (d & 7);
+}
+
+kv_status_t kv_pool_set_poison(kv_pool_t* p, int on) {
+  if (p == nullptr) return KV_ERR_INVALID;
+  p->poison = on != 0;
+  return KV_OK;
+}
+
+kv_status_t kv_alloc(kv_pool_t* p, int n, int* out_page_ids) {
+  if (p == nullptr || n < 0 || (n > 0 && out_page_ids == nullptr)) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(p->mu);
+  if ((size_t)n > p->free_stack.size()) return KV_ERR_OOM;
+  for (int i = 0; i < n; ++i) {
+    const int id = p->free_stack.back();
+    p->free_stack.pop_back();
+    p->allocated[id] = 1;
+    out_page_ids[i] = id;
+  }
+  return KV_OK;
+}
+
+static kv_status_t release_pages(kv_pool_t* p, const int* ids, int n, bool evict) {
+  if (p == nullptr || n < 0 || (n > 0 && ids == nullptr)) return KV_ERR_INVALID;
+  {
+    std::lock_guard<std::mutex> g(p->mu);
+    if (++p->mark_epoch == 0) {  // epoch wrapped: clear the marks
+      std::fill(p->mark.begin(), p->mark.end(), 0u);
+      p->mark_epoch = 1;
+    }
+    for (int i = 0; i < n; ++i) {
+      const int id = ids[i];
+      if (id < 0 || id >= p->num_pages || !p->allocated[id] || p->mark[id] == p->mark_epoch)
+        return KV_ERR_NOT_ALLOCATED;  // nothing has been changed yet
+      p->mark[id] = p->mark_epoch;
+    }
+    for (int i = 0; i < n; ++i) {
+      p->allocated[ids[i]] = 0;
+      p->free_stack.push_back(ids[i]);
+    }
+    if (evict) p->evicted_total += n;
+  }
+  if (evict && p->poison && n > 0) {
+    KV_CUDA_OK(cudaMemcpy(p->d_scratch_ids, ids, sizeof(int) * (size_t)n, cudaMemcpyHostToDevice));
+    poison_kernel<<<n < 1184 ? n : 1184, 256>>>(p->view(), p->d_scratch_ids, n);
+    count_launch();
+    KV_CUDA_OK(cudaGetLastError());
+    KV_CUDA_OK(cudaDeviceSynchronize());
+  }
+  return KV_OK;
+}
+
+kv_status_t kv_free(kv_pool_t* p, const int* page_ids, int n) { return release_pages(p, page_ids, n, false); }
+kv_status_t kv_evict(kv_pool_t* p, const int* page_ids, int n) { return release_pages(p, page_ids, n, true); }
+
+kv_status_t kv_append(kv_pool_t* p, const void* k_new, const void* v_new, const int* cu_new, const int* start_pos,
+                      const int* seg_row, const int* block_tables, int max_pages, int n_segments, int total_new,
+                      void* stream) {
+  if (p == nullptr || n_segments < 0 || total_new < 0 || max_pages < 0) return KV_ERR_INVALID;
+  if (n_segments == 0 || total_new == 0) return KV_OK;
+  if (k_new == nullptr || v_new == nullptr || cu_new == nullptr || start_pos == nullptr || block_tables == nullptr)
+    return KV_ERR_INVALID;
+  if ((((uintptr_t)k_new) | ((uintptr_t)v_new)) & 15) return KV_ERR_INVALID;
+  const int64_t chunks = (int64_t)total_new * p->n_kv_heads * (p->head_dim >> 3);
+  append_kernel<<<grid_for(chunks, 256), 256, 0, (cudaStream_t)stream>>>(
+      p->view(), (const uint4*)k_new, (const uint4*)v_new, cu_new, start_pos, seg_row, block_tables, max_pages,
+      n_segments, total_new);
+  count_launch();
+  KV_CUDA_OK(cudaGetLastError());
+  return KV_OK;
+}
+
+kv_status_t kv_gather(kv_pool_t* p, const int* block_table_row, int len, void* k_out, void* v_out, void* stream) {
+  if (p == nullptr || len < 0) return KV_ERR_INVALID;
+  if (len == 0) return KV_OK;
+  if (block_table_row == nullptr || k_out == nullptr || v_out == nullptr) return KV_ERR_INVALID;
+  if ((((uintptr_t)k_out) | ((uintptr_t)v_out)) & 15) return KV_ERR_INVALID;
+  const int64_t chunks = (int64_t)len * p->n_kv_heads * (p->head_dim >> 3);
+  gather_kernel<<<grid_for(chunks, 256), 256, 0, (cudaStream_t)stream>>>(p->view(), block_table_row, len,
+                                                                         (uint4*)k_out, (uint4*)v_out);
+  count_launch();
+  KV_CUDA_OK(cudaGetLastError());
+  return KV_OK;
+}
+
+kv_status_t kv_last_async_status(kv_pool_t* p) {
+  if (p == nullptr) return KV_ERR_INVALID;
+  int code = 0;
+  KV_CUDA_OK(cudaDeviceSynchronize());
+  KV_CUDA_OK(cudaMemcpy(&code, p->d_status, sizeof(int), cudaMemcpyDeviceToHost));
+  if (code != 0) KV_CUDA_OK(cudaMemset(p->d_status, 0, sizeof(int)));
+  return (kv_status_t)code;
+}
+
+kv_status_t kv_check_batch(kv_pool_t* p, const int* block_tables, int max_pages, const int* lens, int batch,
+                           void* stream) {
+  if (p == nullptr || batch < 0 || max_pages < 0) return KV_ERR_INVALID;
+  if (batch == 0) return KV_OK;
+  if (block_tables == nullptr || lens == nullptr) return KV_ERR_INVALID;
+  check_batch_kernel<<<batch < 1184 ? batch : 1184, 128, 0, (cudaStream_t)stream>>>(p->view(), block_tables,
+                                                                                  max_pages, lens, batch);
+  count_launch();
+  KV_CUDA_OK(cudaGetLastError());
+  KV_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+  return kv_last_async_status(p);
+}
+
+int64_t kvattn_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+}  // extern "C"

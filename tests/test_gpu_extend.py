@@ -1,0 +1,116 @@
+"""attn_extend through the C ABI against the oracle: edge cases, the reuse invariant, aliasing."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_23815_b200 import kvattn, synth
+from harness import Batch, DualPool, assert_close, run_extend
+
+pytestmark = pytest.mark.gpu
+IMPLS = [1, 2]   # 1 = small-tile kernel, 2 = tcgen05 kernel
+
+
+def _skip_if_no_tc(impl, geom):
+    if impl == 2:
+        dp = DualPool(geom, 4, seed=0, with_oracle=False)
+        try:
+            q = torch.zeros((1, geom.n_q_heads, geom.head_dim), dtype=torch.bfloat16, device="cuda")
+            z = torch.zeros(1, dtype=torch.int32, device="cuda")
+            kvattn.kvattn_set_extend_impl(2)
+            try:
+                kvattn.attn_extend(dp.pool, q, torch.tensor([0, 0], dtype=torch.int32, device="cuda"),
+                                   torch.zeros((1, 1), dtype=torch.int32, device="cuda"), z, z, 1, 1, 1.0,
+                                   torch.empty_like(q), torch.empty((1, geom.n_q_heads), device="cuda"),
+                                   torch.empty(1 << 20, dtype=torch.uint8, device="cuda"))
+            except kvattn.KvError as e:
+                if e.status == kvattn.KV_ERR_UNSUPPORTED:
+                    pytest.skip("tensor-core extend kernel does not support this shape")
+                raise
+            finally:
+                kvattn.kvattn_set_extend_impl(0)
+        finally:
+            dp.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("hq,hkv,d", [(4, 2, 64), (32, 8, 128), (8, 1, 128), (4, 4, 64), (16, 2, 128)])
+def test_extend_edge_cases(impl, hq, hkv, d):
+    geom = synth.Geometry(hq, hkv, d)
+    _skip_if_no_tc(impl, geom)
+    P = [0, 1, 15, 16, 17, 31, 32, 0, 100, 5, 130]
+    E = [1, 2, 15, 16, 17, 33, 1, 70, 0, 129, 300]
+    dp = DualPool(geom, 256, seed=200 + hq + d)
+    b = Batch(dp, [p + e for p, e in zip(P, E)])
+    b.write([(i, 0, P[i]) for i in range(len(P))])                     # upstream operator's prefill
+    b.write([(i, P[i], P[i] + E[i]) for i in range(len(P))])           # downstream suffix
+    res = run_extend(dp, b, P, E, impl=impl)
+    assert_close(res, f"extend impl{impl} {hq}/{hkv}/{d}")
+    assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+    dp.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_tiny_config_reuse_equals_from_scratch_prefill(impl):
+    # Config "tiny": 8 tuples, P ~ U[32,128], E ~ U[16,48], 256-page pool, random placement.
+    w = synth.WORKLOADS["tiny"]
+    _skip_if_no_tc(impl, w.geom)
+    ext, _ = synth.draw_lengths(w)
+    P, E = [p for p, _ in ext], [e for _, e in ext]
+    dp = DualPool(w.geom, w.num_pages, seed=w.seed)
+    reuse = Batch(dp, [p + e for p, e in ext])
+    reuse.write([(i, 0, P[i]) for i in range(len(P))])
+    reuse.write([(i, P[i], P[i] + E[i]) for i in range(len(P))])
+    r = run_extend(dp, reuse, P, E, impl=impl)
+    assert_close(r, "tiny reuse")
+    scratch = Batch(dp, [p + e for p, e in ext])                       # same uids -> same values, new pages
+    scratch.write([(i, 0, P[i] + E[i]) for i in range(len(P))])
+    f = run_extend(dp, scratch, [0] * len(P), [p + e for p, e in ext], impl=impl)
+    assert_close(f, "tiny from-scratch")
+    # last E rows of the from-scratch prefill == the reuse run (both within tolerance of the same oracle rows)
+    worst_o = worst_l = 0.0
+    for i in range(len(P)):
+        a0, a1 = r["cu"][i], r["cu"][i + 1]
+        b0 = f["cu"][i] + P[i]
+        assert np.max(np.abs(r["o_ref"][a0:a1] - f["o_ref"][b0:b0 + E[i]])) < 1e-12
+        worst_o = max(worst_o, float(np.max(np.abs(r["o"][a0:a1] - f["o"][b0:b0 + E[i]]))))
+        worst_l = max(worst_l, float(np.max(np.abs(r["lse"][a0:a1] - f["lse"][b0:b0 + E[i]]))))
+    assert worst_o <= 2e-2 and worst_l <= 1e-3
+    dp.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_shared_prefix_fan_out(impl):
+    # A join's children share the parent's prefix pages (full blocks only) and append private suffixes.
+    geom = synth.Geometry(8, 2, 128)
+    _skip_if_no_tc(impl, geom)
+    dp = DualPool(geom, 128, seed=31)
+    fan, P, E = 17, 208, [5 + (3 * c) % 30 for c in range(17)]
+    parent = Batch(dp, [P])
+    parent.write([(0, 0, P)])
+    kids = Batch(dp, E, uid0=100)                                       # private suffix pages only
+    kids.rows = [parent.rows[0] + r for r in kids.rows]                 # alias the parent's pages
+    segs, ks, vs = [], [], []
+    for c in range(fan):
+        k, v = kids.kv(c, P, P + E[c])
+        segs.append((c, P)); ks.append(k); vs.append(v)
+    dp.append(kids.rows, segs, ks, vs)
+    res = run_extend(dp, kids, [P] * fan, E, impl=impl)
+    assert_close(res, "fan-out")
+    dp.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_extend_bit_determinism_and_placement_invariance(impl):
+    geom = synth.Geometry(32, 8, 128)
+    _skip_if_no_tc(impl, geom)
+    P, E = [300, 17, 0], [40, 129, 65]
+    outs = []
+    for seed_perm in (1, 1, 2):
+        dp = DualPool(geom, 128, seed=77)
+        dp.placement = synth.page_permutation(seed_perm, 128).tolist()
+        b = Batch(dp, [p + e for p, e in zip(P, E)])
+        b.write([(i, 0, P[i] + E[i]) for i in range(3)])
+        outs.append(run_extend(dp, b, P, E, impl=impl, oracle=False))
+        dp.close()
+    for o in outs[1:]:
+        assert np.array_equal(outs[0]["o_bits"], o["o_bits"]) and np.array_equal(outs[0]["lse_raw"], o["lse_raw"])
