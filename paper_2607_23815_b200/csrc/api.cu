@@ -60,7 +60,7 @@ kv_status_t attn_extend(kv_pool_t* p, const void* q, int n_q_heads, const int* c
   if ((((uintptr_t)q) | ((uintptr_t)out)) & 15) return KV_ERR_INVALID;
   if (max_total_len < max_extend_len || max_total_len > (int64_t)max_pages * kPageSize) return KV_ERR_INVALID;
   const int impl = g_extend_impl.load();
-  const bool tc_ok = extend_tc_supported(p, n_q_heads);
+  const bool tc_ok = extend_tc_supported(p, n_q_heads) && scale > 0.f;  // the tensor-core kernel folds a positive scale into the row maximum
   if (impl == 2 && !tc_ok) return KV_ERR_UNSUPPORTED;
   if (impl == 2 || (impl == 0 && tc_ok)) {
     return launch_extend_tc(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,

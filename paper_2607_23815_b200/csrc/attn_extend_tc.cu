@@ -1,14 +1,583 @@
-// Tensor-core extend attention (tcgen05 / TMEM).  Placeholder translation unit until the kernel lands:
-// reports "not supported" so that attn_extend selects the small-tile kernel.
+// Tensor-core extend attention for sm_100a: suffix queries over reused prefix pages.
+//
+// Work item = (sequence, KV head, pair of 128-row query tiles).  The rows of a tile are the
+// (suffix token, query head of the KV head's group) pairs, token-major, so the G query heads that
+// share a KV head share every K/V tile that is brought on chip (GQA) and the causal diagonal is
+// only 128/G tokens wide.  One persistent CTA per SM walks a cost-sorted item list.
+//
+// Roles (warp-specialised, 12 warps):
+//   warp 0      producer: per 128-token KV tile, one 1-D bulk copy per 16-token page block
+//               (the pool keeps blocks in the MMA's 128-byte-swizzle operand layout) into a ring of
+//               shared-memory stages; completion is signalled on mbarriers.
+//   warp 1      MMA issuer: S = Q K^T and O += P V on tcgen05 with accumulators in tensor memory;
+//               P is read straight from tensor memory (it overwrites S in place).
+//   warps 4-7   softmax of query tile 0: one thread per row (= TMEM lane): masks, running max and
+//   warps 8-11  sum, exp2, P as bf16 back to TMEM, lazy rescale of O, final normalise + store.
+// The two query tiles ping-pong: while one tile's softmax runs, the tensor core works on the other.
+// All waits are bounded; on expiry the CTA records KV_ERR_TIMEOUT, drains its copies, frees its
+// tensor memory and returns.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace kvattn {
+using namespace ptx;
 
-size_t extend_tc_workspace_bytes(int, int, int, int, int) { return 0; }
-bool extend_tc_supported(const kv_pool_t*, int) { return false; }
-kv_status_t launch_extend_tc(kv_pool_t*, const void*, int, const int*, const int*, int, const int*, const int*, int,
-                             int, int, int, float, void*, float*, void*, size_t, cudaStream_t) {
-  return KV_ERR_UNSUPPORTED;
+constexpr int kTcThreads = 384;
+constexpr int kPlanBuckets = 2048;
+constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more than this
+
+struct TcArgs {
+  PoolView pool;
+  const __nv_bfloat16* q;
+  const int* cu_q;
+  const int* block_tables;
+  int max_pages;
+  const int* prefix_lens;
+  const int* extend_lens;
+  int batch, n_q_heads, group, lg_group;
+  float scale_log2;
+  __nv_bfloat16* out;
+  float* lse;
+  const int2* items;   // (seq, tile pair), cost-sorted
+  const int* n_items;  // number of valid entries in items
+};
+
+// ------------------------------------------------------------------------------------------
+// Plan: list the (sequence, tile pair) entries that have rows, heaviest first (counting sort on
+// the number of KV tile steps).  Only the order of execution depends on it, never a result.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int entry_steps(int P, int E, int tp, int lg) {
+  int steps = 0;
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int r_lo = tp * 256 + t * 128;
+    const int tok_lo = r_lo >> lg;
+    if (tok_lo >= E) break;
+    const int tok_hi = min(E - 1, (r_lo + 127) >> lg);
+    steps += (P + tok_hi + 1 + 127) >> 7;
+  }
+  return steps;
+}
+
+__global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restrict__ prefix_lens,
+                                                              const int* __restrict__ extend_lens, int batch,
+                                                              int max_tp, int lg, int max_steps, int capacity,
+                                                              int2* __restrict__ items, int* __restrict__ n_items) {
+  __shared__ int hist[kPlanBuckets];
+  __shared__ int total;
+  for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
+  __syncthreads();
+  const int64_t n = (int64_t)batch * max_tp;
+  auto key_of = [&](int steps) {
+    const int64_t k = max_steps < kPlanBuckets ? steps : (int64_t)steps * (kPlanBuckets - 1) / max_steps;
+    return (int)min((int64_t)(kPlanBuckets - 1), k);
+  };
+  for (int64_t e = threadIdx.x; e < n; e += blockDim.x) {
+    const int seq = (int)(e / max_tp), tp = (int)(e % max_tp);
+    const int P = __ldg(prefix_lens + seq), E = __ldg(extend_lens + seq);
+    if (P < 0 || E <= 0) continue;
+    const int steps = entry_steps(P, E, tp, lg);
+    if (steps > 0) atomicAdd(&hist[key_of(steps)], 1);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {  // exclusive prefix, heaviest bucket first
+    int run = 0;
+    for (int k = kPlanBuckets - 1; k >= 0; --k) {
+      const int c = hist[k];
+      hist[k] = run;
+      run += c;
+    }
+    total = run;
+    *n_items = min(run, capacity);
+  }
+  __syncthreads();
+  for (int64_t e = threadIdx.x; e < n; e += blockDim.x) {
+    const int seq = (int)(e / max_tp), tp = (int)(e % max_tp);
+    const int P = __ldg(prefix_lens + seq), E = __ldg(extend_lens + seq);
+    if (P < 0 || E <= 0) continue;
+    const int steps = entry_steps(P, E, tp, lg);
+    if (steps > 0) {
+      const int pos = atomicAdd(&hist[key_of(steps)], 1);
+      if (pos < capacity) items[pos] = make_int2(seq, tp);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+template <int D>
+struct TcCfg {
+  static constexpr int kTileBytes = 128 * D * 2;   // a 128-row tile of Q, K or V
+  static constexpr int kBlockBytes = 16 * D * 2;   // one (page, head) block
+  static constexpr int kStages = D == 128 ? 5 : 8;
+  static constexpr uint32_t kGroupStride = D * 16;  // bytes between 8-token groups inside the K/V tiles
+  static constexpr int kHalves = D / 64;
+  static constexpr int kQHalfStride = 128 * 128;    // Q tile: [half][row][128 B]
+};
+
+template <int D>
+struct __align__(1024) TcSmem {
+  unsigned char q[2][TcCfg<D>::kTileBytes];
+  unsigned char kv[TcCfg<D>::kStages][TcCfg<D>::kTileBytes];
+  unsigned long long kv_full[TcCfg<D>::kStages], kv_empty[TcCfg<D>::kStages];
+  unsigned long long q_full[2], s_full[2], p_full[2], o_full[2];
+  uint32_t tmem_base;
+  int abort_flag;
+};
+
+struct Item {
+  int seq, kvh, tp, P, E, row0;
+  int n_kv[2];   // KV tile steps of the two query tiles (0 = tile has no rows)
+  int ld_tiles;  // KV tiles the producer brings in
+  int kv_end;    // keys the item can see at most
+};
+
+__device__ __forceinline__ bool fetch_item(const TcArgs& a, int k, int n_total, Item& it) {
+  if (k >= n_total) return false;
+  const int Hkv = a.pool.n_kv_heads;
+  const int2 e = __ldg(a.items + k / Hkv);
+  it.seq = e.x;
+  it.tp = e.y;
+  it.kvh = k % Hkv;
+  it.P = __ldg(a.prefix_lens + it.seq);
+  it.E = __ldg(a.extend_lens + it.seq);
+  it.row0 = __ldg(a.cu_q + it.seq);
+  it.kv_end = 0;
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int r_lo = it.tp * 256 + t * 128;
+    const int tok_lo = r_lo >> a.lg_group;
+    if (tok_lo >= it.E) {
+      it.n_kv[t] = 0;
+    } else {
+      const int tok_hi = min(it.E - 1, (r_lo + 127) >> a.lg_group);
+      it.n_kv[t] = (it.P + tok_hi + 1 + 127) >> 7;
+      it.kv_end = it.P + tok_hi + 1;
+    }
+  }
+  it.ld_tiles = max(it.n_kv[0], it.n_kv[1]);
+  // a sequence longer than its block-table row can describe is skipped and reported
+  if (it.P + it.E > a.max_pages * kPageSize) {
+    it.n_kv[0] = it.n_kv[1] = it.ld_tiles = 0;
+    return true;
+  }
+  return true;
+}
+
+// item sequence of one CTA: boustrophedon over the sorted list, so that heavy and light items alternate
+__device__ __forceinline__ int item_index(int round) {
+  return (round & 1) ? round * gridDim.x + (gridDim.x - 1 - blockIdx.x) : round * gridDim.x + blockIdx.x;
+}
+
+template <int D>
+__global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcArgs a) {
+  using Cfg = TcCfg<D>;
+  extern __shared__ unsigned char smem_raw[];
+  TcSmem<D>& sm = *reinterpret_cast<TcSmem<D>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  volatile int* abortp = &sm.abort_flag;
+
+  if (tid == 0) {
+    sm.abort_flag = 0;
+    for (int s = 0; s < Cfg::kStages; ++s) {
+      mbar_init(smem_u32(&sm.kv_full[s]), 1);
+      mbar_init(smem_u32(&sm.kv_empty[s]), 1);
+    }
+    for (int t = 0; t < 2; ++t) {
+      mbar_init(smem_u32(&sm.q_full[t]), 128);
+      mbar_init(smem_u32(&sm.s_full[t]), 1);
+      mbar_init(smem_u32(&sm.p_full[t]), 128);
+      mbar_init(smem_u32(&sm.o_full[t]), 1);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&sm.tmem_base), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = sm.tmem_base;
+  const int n_total = __ldg(a.n_items) * a.pool.n_kv_heads;
+  const int Hkv = a.pool.n_kv_heads;
+
+  if (warp == 0) {
+    // =============================== producer =============================================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    const char* kpool = reinterpret_cast<const char*>(a.pool.k);
+    const char* vpool = reinterpret_cast<const char*>(a.pool.v);
+    uint32_t loads = 0;  // stage loads issued so far (ring position)
+    bool ok = true;
+    for (int round = 0; ok; ++round) {
+      Item it;
+      if (!fetch_item(a, item_index(round), n_total, it)) break;
+      const int* bt = a.block_tables + (int64_t)it.seq * a.max_pages;
+      const size_t head_off = (size_t)it.kvh * Cfg::kBlockBytes;
+      for (int j = 0; j < it.ld_tiles && ok; ++j) {
+        const int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
+        int page = 0;
+        if (lane < np) {
+          page = __ldg(bt + j * 8 + lane);
+          if ((unsigned)page >= (unsigned)a.pool.num_pages) {
+            report(a.pool.status, KV_ERR_BOUNDS);
+            page = 0;
+          }
+        }
+        const size_t src_off = ((size_t)page * Hkv) * Cfg::kBlockBytes + head_off;
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {  // 0: K tile, 1: V tile
+          const uint32_t s = loads % Cfg::kStages, par = (loads / Cfg::kStages) & 1;
+          const uint32_t full = smem_u32(&sm.kv_full[s]);
+          if (lane == 0) {
+            ok = mbar_wait(smem_u32(&sm.kv_empty[s]), par ^ 1, abortp);
+            if (ok) mbar_arrive_expect_tx(full, (uint32_t)np * Cfg::kBlockBytes);
+          }
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          if (lane < np)
+            bulk_g2s(smem_u32(sm.kv[s]) + lane * Cfg::kBlockBytes, (which ? vpool : kpool) + src_off, Cfg::kBlockBytes,
+                     full);
+          ++loads;
+        }
+      }
+    }
+    if (!ok && lane == 0) {
+      // give copies that were already issued time to land before the CTA's shared memory goes away
+      const uint32_t first = loads > (uint32_t)Cfg::kStages ? loads - Cfg::kStages : 0;
+      for (uint32_t i = first; i < loads; ++i) {
+        const uint32_t s = i % Cfg::kStages, par = (i / Cfg::kStages) & 1;
+        const uint64_t t0 = globaltimer_ns();
+        while (!mbar_try_wait(smem_u32(&sm.kv_full[s]), par) && globaltimer_ns() - t0 < 100000000ull) {
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // =============================== MMA issuer ===========================================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);  // S[128 x 128 keys] = Q (K-major) x K (K-major)
+    constexpr uint32_t idesc_o = idesc_bf16(128, D, 0, 1);    // O[128 x D] += P (TMEM) x V (MN-major)
+    uint32_t loads = 0;                 // ring position, mirrors the producer
+    uint32_t steps[2] = {0, 0};         // softmax steps per tile so far (phase of s_full / p_full)
+    uint32_t items_done[2] = {0, 0};    // items per tile so far (phase of q_full / o_full)
+    bool ok = true;
+    for (int round = 0; ok; ++round) {
+      Item it;
+      if (!fetch_item(a, item_index(round), n_total, it)) break;
+      if (it.ld_tiles == 0) continue;
+      if (lane == 0) {
+        const bool act1 = it.n_kv[1] > 0;
+        ok = mbar_wait(smem_u32(&sm.q_full[0]), items_done[0] & 1, abortp);
+        if (ok && act1) ok = mbar_wait(smem_u32(&sm.q_full[1]), items_done[1] & 1, abortp);
+        tc_fence_after_sync();
+        auto issue_s = [&](int t, uint32_t stage) {
+          const uint32_t qb = smem_u32(sm.q[t]), kb = smem_u32(sm.kv[stage]);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            const uint64_t ad = smem_desc_sw128(qb + (ks >> 2) * Cfg::kQHalfStride + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = smem_desc_sw128(kb + (ks >> 2) * 1024 + (ks & 3) * 32, 16, Cfg::kGroupStride);
+            mma_ss(tmem + t * 128, ad, bd, idesc_s, ks > 0);
+          }
+          mma_commit(smem_u32(&sm.s_full[t]));
+        };
+        auto issue_pv = [&](int t, uint32_t stage, int np, bool first) {
+          const uint32_t vb = smem_u32(sm.kv[stage]);
+          for (int p = 0; p < np; ++p) {
+            const uint64_t bd = smem_desc_sw128(vb + p * Cfg::kBlockBytes, 1024, Cfg::kGroupStride);
+            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + p * 8, bd, idesc_o, !(first && p == 0));
+          }
+        };
+        // first K tile: S of both query tiles
+        uint32_t ks_stage = loads % Cfg::kStages;
+        ok = ok && mbar_wait(smem_u32(&sm.kv_full[ks_stage]), (loads / Cfg::kStages) & 1, abortp);
+        if (ok) {
+          tc_fence_after_sync();
+          issue_s(0, ks_stage);
+          if (act1) issue_s(1, ks_stage);
+          mma_commit(smem_u32(&sm.kv_empty[ks_stage]));
+        }
+        ++loads;
+        for (int j = 0; j < it.ld_tiles && ok; ++j) {
+          const int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
+          const uint32_t v_stage = loads % Cfg::kStages;
+          ok = mbar_wait(smem_u32(&sm.kv_full[v_stage]), (loads / Cfg::kStages) & 1, abortp);
+          ++loads;
+          if (!ok) break;
+          // slots past the end of the sequence may hold anything (NaN included): zero them, because the
+          // MMA multiplies them with P = 0
+          const int seq_len = it.P + it.E;
+          const int tail_lo = seq_len - j * 128;
+          if (tail_lo < np * 16) {
+            for (int r = max(tail_lo, 0); r < np * 16; ++r) {
+              unsigned char* rowp = sm.kv[v_stage] + (r >> 3) * Cfg::kGroupStride + (r & 7) * 128;
+#pragma unroll
+              for (int h = 0; h < Cfg::kHalves; ++h)
+#pragma unroll
+                for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(rowp + h * 1024 + c * 16) = make_uint4(0, 0, 0, 0);
+            }
+            fence_proxy_async_smem();
+          }
+          tc_fence_after_sync();
+          const bool more = j + 1 < it.ld_tiles;
+          uint32_t k_stage = 0;
+          if (more) {
+            k_stage = loads % Cfg::kStages;
+            ok = mbar_wait(smem_u32(&sm.kv_full[k_stage]), (loads / Cfg::kStages) & 1, abortp);
+            ++loads;
+            if (!ok) break;
+            tc_fence_after_sync();
+          }
+#pragma unroll
+          for (int t = 0; t < 2; ++t) {
+            if (j >= it.n_kv[t]) continue;
+            ok = mbar_wait(smem_u32(&sm.p_full[t]), steps[t] & 1, abortp);
+            ++steps[t];
+            if (!ok) break;
+            tc_fence_after_sync();
+            issue_pv(t, v_stage, np, j == 0);
+            if (j + 1 < it.n_kv[t]) {
+              issue_s(t, k_stage);
+            } else {
+              mma_commit(smem_u32(&sm.o_full[t]));
+            }
+          }
+          if (!ok) break;
+          mma_commit(smem_u32(&sm.kv_empty[v_stage]));
+          if (more) mma_commit(smem_u32(&sm.kv_empty[k_stage]));
+        }
+        ++items_done[0];
+        if (act1) ++items_done[1];
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      loads = __shfl_sync(0xffffffffu, loads, 0);
+    }
+  } else if (warp >= 4) {
+    // =============================== softmax / epilogue ===================================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    const int t = (warp - 4) >> 2;                 // query tile of this warpgroup
+    const int w4 = warp & 3;                       // TMEM lane quarter this warp may access
+    const int m = w4 * 32 + lane;                  // row inside the tile
+    const uint32_t lane_base = tmem + ((uint32_t)(w4 * 32) << 16);
+    const uint32_t s_addr = lane_base + t * 128, o_addr = lane_base + 256 + t * 128;
+    const int G = a.group, lg = a.lg_group, Hq = a.n_q_heads;
+    uint32_t steps = 0, items_done = 0;
+    bool ok = true;
+    for (int round = 0; ok; ++round) {
+      Item it;
+      if (!fetch_item(a, item_index(round), n_total, it)) break;
+      if (it.n_kv[t] == 0) continue;
+      // ---- Q tile -> shared memory in the swizzled K-major operand layout (coalesced 16-byte loads)
+      {
+        constexpr int CPR = D / 8, RPI = 32 / CPR;  // chunks per row, rows per iteration of one warp
+#pragma unroll 4
+        for (int i = 0; i < 32 / RPI; ++i) {
+          const int row = w4 * 32 + i * RPI + lane / CPR, chunk = lane % CPR;
+          const int rg = it.tp * 256 + t * 128 + row;
+          const int tok = rg >> lg;
+          uint4 val = make_uint4(0, 0, 0, 0);
+          if (tok < it.E)
+            val = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1))) * D) + chunk);
+          *reinterpret_cast<uint4*>(sm.q[t] + (chunk >> 3) * Cfg::kQHalfStride + (row >> 3) * 1024 + (row & 7) * 128 +
+                                    (((chunk & 7) ^ (row & 7)) << 4)) = val;
+        }
+        fence_proxy_async_smem();
+        mbar_arrive(smem_u32(&sm.q_full[t]));
+      }
+      const int rg = it.tp * 256 + t * 128 + m;
+      const int tok = rg >> lg;
+      const bool valid = tok < it.E;
+      const int limit = valid ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
+      float m_run = -INFINITY, l_run = 0.f;
+
+      for (int j = 0; j < it.n_kv[t] && ok; ++j) {
+        ok = mbar_wait(smem_u32(&sm.s_full[t]), steps & 1, abortp);
+        ++steps;
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t sr[4][32];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr[c]);
+        tmem_wait_ld();
+        const int kv0 = j * 128;
+        float mx = -INFINITY;
+        if (kv0 + 128 <= limit) {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[c][i]));
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+              const float v = (kv0 + c * 32 + i < limit) ? __uint_as_float(sr[c][i]) : -INFINITY;  // select: NaN-safe
+              sr[c][i] = __float_as_uint(v);
+              mx = fmaxf(mx, v);
+            }
+        }
+        mx *= a.scale_log2;
+        const float m_new = fmaxf(m_run, mx);
+        const bool grow = m_new > m_run + kRescaleThreshold;  // also true on the first tile (m_run = -inf)
+        const float m_use = grow ? m_new : m_run;
+        if (j > 0 && __any_sync(0xffffffffu, grow)) {
+          const float alpha = grow ? exp2f(m_run - m_new) : 1.f;
+          l_run *= alpha;
+#pragma unroll
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t orow[32];
+            tmem_ld32(o_addr + c * 32, orow);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) orow[i] = __float_as_uint(__uint_as_float(orow[i]) * alpha);
+            tmem_st32(o_addr + c * 32, orow);
+          }
+        }
+        m_run = m_use;
+        const float neg_m = (m_use == -INFINITY) ? 0.f : -m_use;
+        float lsum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            float p0, p1;
+            const float x0 = fmaf(__uint_as_float(sr[c][2 * i]), a.scale_log2, neg_m);
+            const float x1 = fmaf(__uint_as_float(sr[c][2 * i + 1]), a.scale_log2, neg_m);
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p0) : "f"(x0));
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p1) : "f"(x1));
+            lsum += p0 + p1;
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[i]) : "f"(p1), "f"(p0));
+          }
+          tmem_st16(s_addr + c * 16, pk);  // P overwrites the S columns already held in registers
+        }
+        l_run += lsum;
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(smem_u32(&sm.p_full[t]));
+      }
+      if (!ok) break;
+      // ---- epilogue: O / l -> bf16, LSE
+      ok = mbar_wait(smem_u32(&sm.o_full[t]), items_done & 1, abortp);
+      ++items_done;
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const float inv = 1.f / l_run;
+      const int64_t orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) {
+        uint32_t orow[32];
+        tmem_ld32(o_addr + c * 32, orow);
+        tmem_wait_ld();
+        if (valid) {
+          uint4* dst = reinterpret_cast<uint4*>(a.out + orow_idx * D + c * 32);
+#pragma unroll
+          for (int v4 = 0; v4 < 4; ++v4) {
+            uint32_t w[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const float lo = __uint_as_float(orow[v4 * 8 + 2 * i]) * inv, hi = __uint_as_float(orow[v4 * 8 + 2 * i + 1]) * inv;
+              asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(hi), "f"(lo));
+            }
+            dst[v4] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      if (valid) a.lse[orow_idx] = (m_run + log2f(l_run)) * 0.6931471805599453f;
+      tc_fence_before_sync();
+    }
+  } else {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (tid == 0 && sm.abort_flag != 0) report(a.pool.status, KV_ERR_TIMEOUT);
+  if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// ------------------------------------------------------------------------------------------
+static inline size_t align256(size_t x) { return (x + 255) & ~(size_t)255; }
+
+static int64_t item_capacity(int n_q_heads, int n_kv_heads, int batch, int total_q) {
+  const int G = n_q_heads / n_kv_heads;
+  return (int64_t)total_q * G / 256 + batch + 1;
+}
+
+size_t extend_tc_workspace_bytes(int n_q_heads, int head_dim, int batch, int total_q, int max_total_len) {
+  (void)head_dim; (void)max_total_len;
+  if (batch <= 0 || total_q <= 0) return 0;
+  // n_kv_heads is not known here: G <= 8 bounds the list
+  return 256 + align256(sizeof(int2) * (size_t)((int64_t)total_q * 8 / 256 + batch + 1));
+}
+
+bool extend_tc_supported(const kv_pool_t* p, int n_q_heads) {
+  if (p->head_dim != 64 && p->head_dim != 128) return false;
+  const int g = n_q_heads / p->n_kv_heads;
+  return g == 1 || g == 2 || g == 4 || g == 8;
+}
+
+template <int D>
+static kv_status_t launch_tc(const TcArgs& a, int n_items_bound, cudaStream_t st) {
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0;
+    KV_CUDA_OK(cudaGetDevice(&dev));
+    KV_CUDA_OK(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+  }
+  const size_t smem = sizeof(TcSmem<D>) + 1024;
+  static bool configured = false;
+  if (!configured) {
+    KV_CUDA_OK(cudaFuncSetAttribute(attn_extend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    configured = true;
+  }
+  const int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
+  attn_extend_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(a);
+  count_launch();
+  KV_CUDA_OK(cudaGetLastError());
+  return KV_OK;
+}
+
+kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                             int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                             int max_extend_len, int max_total_len, float scale, void* out, float* lse,
+                             void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  const size_t need = extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch, total_q, max_total_len);
+  if (workspace == nullptr || workspace_bytes < need) return KV_ERR_WORKSPACE;
+  const int G = n_q_heads / p->n_kv_heads;
+  int lg = 0;
+  while ((1 << lg) < G) ++lg;
+  int* n_items = reinterpret_cast<int*>(workspace);
+  int2* items = reinterpret_cast<int2*>(reinterpret_cast<char*>(workspace) + 256);
+  const int64_t capacity = item_capacity(n_q_heads, p->n_kv_heads, batch, total_q);
+  const int max_tp = (int)(((int64_t)max_extend_len * G + 255) / 256);
+  const int max_steps = 2 * ((max_total_len + 127) / 128);
+  extend_tc_plan_kernel<<<1, 1024, 0, st>>>(prefix_lens, extend_lens, batch, max_tp, lg, max_steps, (int)capacity,
+                                            items, n_items);
+  count_launch();
+  KV_CUDA_OK(cudaGetLastError());
+
+  TcArgs a{};
+  a.pool = p->view();
+  a.q = (const __nv_bfloat16*)q;
+  a.cu_q = cu_q;
+  a.block_tables = block_tables;
+  a.max_pages = max_pages;
+  a.prefix_lens = prefix_lens;
+  a.extend_lens = extend_lens;
+  a.batch = batch;
+  a.n_q_heads = n_q_heads;
+  a.group = G;
+  a.lg_group = lg;
+  a.scale_log2 = scale * 1.4426950408889634f;
+  a.out = (__nv_bfloat16*)out;
+  a.lse = lse;
+  a.items = items;
+  a.n_items = n_items;
+  const int64_t bound = (int64_t)batch * max_tp * p->n_kv_heads;
+  const int n_bound = bound > (1 << 30) ? (1 << 30) : (int)bound;
+  if (p->head_dim == 128) return launch_tc<128>(a, n_bound, st);
+  return launch_tc<64>(a, n_bound, st);
 }
 
 }  // namespace kvattn
