@@ -277,13 +277,14 @@ def run_ours(args):
         "clocks": clocks,
     }
 
-    if rank == 0 and world == 1 and not args.headline_only:
-        # ---- CPU oracle on a bounded sample of the same workload ---------------------------
-        n_s = min(args.cpu_sample, len(e.prefix))
-        dt, work, err_o, err_l = cpu_oracle_sample(wl, n_s, "extend")
-        line["cpu_baseline"] = {"value": round(work / dt / 1e12, 6), "unit": "TFLOP/s", "cores": blas_threads(),
-                                "kind": "oracle", "sample": f"first {n_s} of {len(e.prefix)} tuples, {dt:.1f} s",
-                                "max_abs_err_o_vs_gpu": err_o, "max_abs_err_lse_vs_gpu": err_l}
+    if rank == 0 and world == 1:
+        if not args.no_cpu:
+            # ---- CPU oracle on a bounded sample of the same workload -----------------------
+            n_s = min(args.cpu_sample, len(e.prefix))
+            dt, work, err_o, err_l = cpu_oracle_sample(wl, n_s, "extend")
+            line["cpu_baseline"] = {"value": round(work / dt / 1e12, 6), "unit": "TFLOP/s", "cores": blas_threads(),
+                                    "kind": "oracle", "sample": f"first {n_s} of {len(e.prefix)} tuples, {dt:.1f} s",
+                                    "max_abs_err_o_vs_gpu": err_o, "max_abs_err_lse_vs_gpu": err_l}
         wl.close(); del wl
         torch.cuda.empty_cache()
         line.update(extra_measurements(args, dev, peaks, flush))
@@ -301,27 +302,34 @@ def extra_measurements(args, dev, peaks, flush):
     from paper_2607_23815_b200 import kvattn
     from paper_2607_23815_b200.workload import DeviceWorkload
     out = {}
+    sections = set(x for x in args.sections.split(",") if x and x != "none")
     steps, warm = max(5, args.steps), 3
+    if not sections & {"decode", "append"}:
+        return mixed_measurement(args, dev, flush, steps, warm) if "mixed" in sections else out
     # decode
     w = synth.WORKLOADS["decode_8b"]
     wl = DeviceWorkload(w, dev)
     ms, _ = time_steps(lambda _: wl.decode(), steps, warm, flush, 1)
     t = statistics.mean(ms)
     gbs = wl.dec.kv_bytes(w.geom) / (t * 1e-3) / 1e9
-    dt, work, err_o, err_l = cpu_oracle_sample(wl, min(128, len(wl.dec.ctx)), "decode")
+    if args.no_cpu:
+        dt, work, err_o, err_l = float("nan"), float("nan"), None, None
+    else:
+        dt, work, err_o, err_l = cpu_oracle_sample(wl, min(128, len(wl.dec.ctx)), "decode")
     out["decode"] = {"workload": f"{w.name}: {w.n_decode} seqs, ctx U{list(w.ctx_range)}, {w.num_pages}-page pool",
                      "value": round(gbs, 1), "unit": "GB/s", "ms_per_step": round(t, 5), "min_ms": round(min(ms), 5),
                      "roofline": {"bound": "hbm", "kernel": "attn_decode", "achieved": round(gbs, 1),
                                   "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(gbs / peaks["hbm_gbs"], 4),
                                   "peak_source": f"{peaks['source']} (copy)", "frac_of_nominal_8000": round(gbs / 8000.0, 4),
                                   "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
-                     "cpu_baseline": {"value": round(work / dt / 1e9, 4), "unit": "GB/s", "cores": blas_threads(),
-                                      "kind": "oracle", "sample": f"first {min(128, w.n_decode)} of {w.n_decode} sequences, {dt:.1f} s",
-                                      "max_abs_err_o_vs_gpu": err_o, "max_abs_err_lse_vs_gpu": err_l}}
+                     "cpu_baseline": None if args.no_cpu else {
+                         "value": round(work / dt / 1e9, 4), "unit": "GB/s", "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"first {min(128, w.n_decode)} of {w.n_decode} sequences, {dt:.1f} s",
+                         "max_abs_err_o_vs_gpu": err_o, "max_abs_err_lse_vs_gpu": err_l}}
     # bulk append: re-write every decode sequence's K/V (read + write bytes)
     d = wl.dec
     n_tok = sum(d.ctx)
-    if n_tok * w.geom.kv_bytes_per_token < 6 << 30:
+    if "append" in sections and n_tok * w.geom.kv_bytes_per_token < 6 << 30:
         k_all = torch.empty((n_tok, w.geom.n_kv_heads, w.geom.head_dim), dtype=torch.bfloat16, device=dev).normal_()
         v_all = torch.empty_like(k_all).normal_()
         cu = torch.tensor(np.concatenate([[0], np.cumsum(d.ctx)]), dtype=torch.int32, device=dev)
@@ -337,7 +345,15 @@ def extra_measurements(args, dev, peaks, flush):
         del k_all, v_all
     wl.close(); del wl
     torch.cuda.empty_cache()
-    # mixed pipeline step
+    if "mixed" in sections:
+        out.update(mixed_measurement(args, dev, flush, steps, warm))
+    return out
+
+
+def mixed_measurement(args, dev, flush, steps, warm):
+    """One sem_map -> sem_filter pipeline step: extend set and decode set together."""
+    from paper_2607_23815_b200.workload import DeviceWorkload
+    out = {}
     w = synth.WORKLOADS["pipeline_step"]
     wl = DeviceWorkload(w, dev)
     ms_mixed, _ = time_steps(lambda _: wl.mixed(), steps, warm, flush, 1)
@@ -407,7 +423,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=HEADLINE, choices=[k for k, v in synth.WORKLOADS.items() if v.n_extend])
     ap.add_argument("--cpu-sample", type=int, default=64, help="tuples in the CPU-oracle sample")
-    ap.add_argument("--headline-only", action="store_true", help="skip the decode/append/mixed extras")
+    ap.add_argument("--sections", default="decode,append,mixed",
+                    help="extra measurements after the headline: comma list of decode, append, mixed (or 'none')")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle legs (for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":

@@ -108,8 +108,11 @@ kv_status_t kv_evict(kv_pool_t* pool, const int* page_ids /*host*/, int n);
  * ([dev] bf16 [total_new][n_kv_heads][head_dim]) and writes them to token positions
  * start_pos[s] .. of the sequence whose block-table row is seg_row[s] (seg_row NULL: row s).
  * cu_new [dev][n_segments+1], start_pos [dev][n_segments], seg_row [dev][n_segments] or NULL,
- * block_tables [dev][rows][max_pages].  Segments must not overlap each other.  Pure data movement:
- * the stored bits equal the input bits. */
+ * block_tables [dev][rows][max_pages].  Pure data movement: the stored bits equal the input bits.
+ * A segment also clears (to zero bits) the slots that follow its last token in that token's page, so
+ * the tail of a sequence's last page never holds stale NaN/Inf patterns; tokens are therefore appended
+ * to a page in increasing position order, and two segments of one call must not write into the same
+ * page (segments that meet at a page boundary are fine). */
 kv_status_t kv_append(kv_pool_t* pool, const void* k_new, const void* v_new, const int* cu_new,
                       const int* start_pos, const int* seg_row, const int* block_tables, int max_pages,
                       int n_segments, int total_new, void* stream);

@@ -9,8 +9,8 @@
 //   warp 0      producer: per 128-token KV tile, one 1-D bulk copy per 16-token page block
 //               (the pool keeps blocks in the MMA's 128-byte-swizzle operand layout) into a ring of
 //               shared-memory stages; completion is signalled on mbarriers.
-//   warp 1      MMA issuer: S = Q K^T and O += P V on tcgen05 with accumulators in tensor memory;
-//               P is read straight from tensor memory (it overwrites S in place).
+//   warps 1, 2  MMA issuers, one per query tile: S = Q K^T and O += P V on tcgen05 with accumulators in
+//               tensor memory; P is read straight from tensor memory (it overwrites S in place).
 //   warps 4-7   softmax of query tile 0: one thread per row (= TMEM lane): masks, running max and
 //   warps 8-11  sum, exp2, P as bf16 back to TMEM, lazy rescale of O, final normalise + store.
 // The two query tiles ping-pong: while one tile's softmax runs, the tensor core works on the other.
@@ -22,7 +22,7 @@
 namespace kvattn {
 using namespace ptx;
 
-constexpr int kTcThreads = 384;
+constexpr int kTcThreads = 384;  // warp 0: producer, warps 1-3: idle, warps 4-11: two softmax warpgroups
 constexpr int kPlanBuckets = 2048;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more than this
 
@@ -38,7 +38,7 @@ struct TcArgs {
   float scale_log2;
   __nv_bfloat16* out;
   float* lse;
-  const int2* items;   // (seq, tile pair), cost-sorted
+  const int4* items;   // two int4 per entry (see ItemRec), cost-sorted
   const int* n_items;  // number of valid entries in items
 };
 
@@ -59,12 +59,35 @@ __device__ __forceinline__ int entry_steps(int P, int E, int tp, int lg) {
   return steps;
 }
 
+// One entry of the plan: everything a CTA needs to know about a (sequence, tile pair), so that the
+// roles read one 32-byte record per item instead of chasing the length arrays.
+struct ItemRec {
+  int seq, tp, P, E;
+  int row0, n_kv0, n_kv1, kv_end;  // first query row; KV tile steps of the two tiles; keys the item sees at most
+};
+
+__device__ __forceinline__ ItemRec make_item(int seq, int tp, int P, int E, int row0, int lg, int max_pages) {
+  ItemRec r{seq, tp, P, E, row0, 0, 0, 0};
+#pragma unroll
+  for (int t = 0; t < 2; ++t) {
+    const int r_lo = tp * 256 + t * 128;
+    const int tok_lo = r_lo >> lg;
+    if (tok_lo >= E) break;
+    const int tok_hi = min(E - 1, (r_lo + 127) >> lg);
+    (t ? r.n_kv1 : r.n_kv0) = (P + tok_hi + 1 + 127) >> 7;
+    r.kv_end = P + tok_hi + 1;
+  }
+  if (P + E > max_pages * kPageSize) r.n_kv0 = r.n_kv1 = 0;  // longer than its block-table row: skipped (reported by the plan)
+  return r;
+}
+
 __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restrict__ prefix_lens,
-                                                              const int* __restrict__ extend_lens, int batch,
-                                                              int max_tp, int lg, int max_steps, int capacity,
-                                                              int2* __restrict__ items, int* __restrict__ n_items) {
+                                                              const int* __restrict__ extend_lens,
+                                                              const int* __restrict__ cu_q, int batch, int max_tp,
+                                                              int lg, int max_steps, int capacity, int max_pages,
+                                                              int* status, int4* __restrict__ items,
+                                                              int* __restrict__ n_items) {
   __shared__ int hist[kPlanBuckets];
-  __shared__ int total;
   for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const int64_t n = (int64_t)batch * max_tp;
@@ -87,7 +110,6 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
       hist[k] = run;
       run += c;
     }
-    total = run;
     *n_items = min(run, capacity);
   }
   __syncthreads();
@@ -98,9 +120,20 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
     const int steps = entry_steps(P, E, tp, lg);
     if (steps > 0) {
       const int pos = atomicAdd(&hist[key_of(steps)], 1);
-      if (pos < capacity) items[pos] = make_int2(seq, tp);
+      if (pos < capacity) {
+        const ItemRec r = make_item(seq, tp, P, E, __ldg(cu_q + seq), lg, max_pages);
+        if (r.n_kv0 == 0) report(status, KV_ERR_BOUNDS);
+        items[2 * pos] = make_int4(r.seq, r.tp, r.P, r.E);
+        items[2 * pos + 1] = make_int4(r.row0, r.n_kv0, r.n_kv1, r.kv_end);
+      }
     }
   }
+}
+
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
 }
 
 // ------------------------------------------------------------------------------------------
@@ -131,36 +164,45 @@ struct Item {
   int kv_end;    // keys the item can see at most
 };
 
+// Item k of the global list: entry k / Hkv of the plan, KV head k % Hkv.  Returns false past the end.
 __device__ __forceinline__ bool fetch_item(const TcArgs& a, int k, int n_total, Item& it) {
   if (k >= n_total) return false;
   const int Hkv = a.pool.n_kv_heads;
-  const int2 e = __ldg(a.items + k / Hkv);
-  it.seq = e.x;
-  it.tp = e.y;
-  it.kvh = k % Hkv;
-  it.P = __ldg(a.prefix_lens + it.seq);
-  it.E = __ldg(a.extend_lens + it.seq);
-  it.row0 = __ldg(a.cu_q + it.seq);
-  it.kv_end = 0;
-#pragma unroll
-  for (int t = 0; t < 2; ++t) {
-    const int r_lo = it.tp * 256 + t * 128;
-    const int tok_lo = r_lo >> a.lg_group;
-    if (tok_lo >= it.E) {
-      it.n_kv[t] = 0;
-    } else {
-      const int tok_hi = min(it.E - 1, (r_lo + 127) >> a.lg_group);
-      it.n_kv[t] = (it.P + tok_hi + 1 + 127) >> 7;
-      it.kv_end = it.P + tok_hi + 1;
-    }
-  }
+  const int e = k / Hkv;
+  const int4 r0 = __ldg(a.items + 2 * e), r1 = __ldg(a.items + 2 * e + 1);
+  it.seq = r0.x; it.tp = r0.y; it.P = r0.z; it.E = r0.w;
+  it.row0 = r1.x; it.n_kv[0] = r1.y; it.n_kv[1] = r1.z; it.kv_end = r1.w;
+  it.kvh = k - e * Hkv;
   it.ld_tiles = max(it.n_kv[0], it.n_kv[1]);
-  // a sequence longer than its block-table row can describe is skipped and reported
-  if (it.P + it.E > a.max_pages * kPageSize) {
-    it.n_kv[0] = it.n_kv[1] = it.ld_tiles = 0;
-    return true;
-  }
   return true;
+}
+
+// Operand descriptors differ only in their low word (start address >> 4 plus the leading-dimension
+// offset field); the high word is a constant.  Issuing an MMA then costs one add, so a single thread
+// keeps the tensor pipe fed.
+__device__ __forceinline__ uint64_t make_desc(uint32_t hi, uint32_t lo) { return ((uint64_t)hi << 32) | lo; }
+
+// S[128 rows x 128 keys] = Q_t (K-major, shared) x K_stage (K-major, shared); q_lo / k_lo: low descriptor words
+template <int D>
+__device__ __forceinline__ void issue_s_mmas(uint32_t s_tmem, uint32_t q_lo, uint32_t k_lo) {
+  constexpr uint32_t kHiQ = (1024u >> 4) | (1u << 14) | (2u << 29);        // SBO 1024, sm_100 descriptor, 128B swizzle
+  constexpr uint32_t kHiK = ((uint32_t)(D * 16) >> 4) | (1u << 14) | (2u << 29);  // SBO = 8-token group stride
+  constexpr uint32_t idesc = idesc_bf16(128, 128, 0, 0);
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks)
+    mma_ss(s_tmem, make_desc(kHiQ, q_lo + (ks >> 2) * 1024 + (ks & 3) * 2), make_desc(kHiK, k_lo + (ks >> 2) * 64 + (ks & 3) * 2),
+           idesc, ks > 0);
+}
+
+// O[128 rows x D] (+)= P (bf16 in tensor memory) x V_stage (MN-major, shared), one MMA per 16-token page
+template <int D>
+__device__ __forceinline__ void issue_pv_mmas(uint32_t o_tmem, uint32_t p_tmem, uint32_t v_lo, int np, bool first) {
+  constexpr uint32_t kHiV = ((uint32_t)(D * 16) >> 4) | (1u << 14) | (2u << 29);
+  constexpr uint32_t idesc = idesc_bf16(128, D, 0, 1);
+  mma_ts(o_tmem, p_tmem, make_desc(kHiV, v_lo), idesc, first ? 0u : 1u);
+#pragma unroll
+  for (int p = 1; p < 8; ++p)
+    if (p < np) mma_ts(o_tmem, p_tmem + p * 8, make_desc(kHiV, v_lo + p * (D * 2)), idesc, 1u);
 }
 
 // item sequence of one CTA: boustrophedon over the sorted list, so that heavy and light items alternate
@@ -183,14 +225,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       mbar_init(smem_u32(&sm.kv_empty[s]), 1);
     }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(smem_u32(&sm.q_full[t]), 128);
-      mbar_init(smem_u32(&sm.s_full[t]), 1);
-      mbar_init(smem_u32(&sm.p_full[t]), 128);
-      mbar_init(smem_u32(&sm.o_full[t]), 1);
+      mbar_init(smem_u32(&sm.q_full[t]), 128);  // every softmax thread stored its part of the Q tile
+      mbar_init(smem_u32(&sm.s_full[t]), 1);    // tensor core finished S (and everything issued before it)
+      mbar_init(smem_u32(&sm.p_full[t]), 128);  // every softmax thread wrote its row of P
+      mbar_init(smem_u32(&sm.o_full[t]), 1);    // tensor core finished the item's last PV
     }
     fence_mbar_init();
   }
-  if (warp == 1) {
+  if (warp == 0) {
     tmem_alloc(smem_u32(&sm.tmem_base), 512);
     tmem_relinquish();
   }
@@ -203,14 +245,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
 
   if (warp == 0) {
     // =============================== producer =============================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     const char* kpool = reinterpret_cast<const char*>(a.pool.k);
     const char* vpool = reinterpret_cast<const char*>(a.pool.v);
     uint32_t loads = 0;  // stage loads issued so far (ring position)
     bool ok = true;
-    for (int round = 0; ok; ++round) {
-      Item it;
-      if (!fetch_item(a, item_index(round), n_total, it)) break;
+    Item nxt;
+    bool has_nxt = fetch_item(a, item_index(0), n_total, nxt);
+    for (int round = 0; ok && has_nxt; ++round) {
+      const Item it = nxt;
+      has_nxt = fetch_item(a, item_index(round + 1), n_total, nxt);  // next record is in flight during this item
       const int* bt = a.block_tables + (int64_t)it.seq * a.max_pages;
       const size_t head_off = (size_t)it.kvh * Cfg::kBlockBytes;
       for (int j = 0; j < it.ld_tiles && ok; ++j) {
@@ -253,70 +297,46 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
     }
   } else if (warp == 1) {
     // =============================== MMA issuer ===========================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
-    constexpr uint32_t idesc_s = idesc_bf16(128, 128, 0, 0);  // S[128 x 128 keys] = Q (K-major) x K (K-major)
-    constexpr uint32_t idesc_o = idesc_bf16(128, D, 0, 1);    // O[128 x D] += P (TMEM) x V (MN-major)
+    // One thread issues every MMA of the CTA.  Per KV tile j and query tile t:  O_t (+)= P_t V(j) as soon as
+    // the softmax warps have written P_t, then S_t = Q_t K(j+1)^T into the columns P_t occupied (the tensor
+    // core runs MMAs in issue order), so the other tile's MMAs fill the time this tile's softmax takes.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+    const uint32_t q_lo0 = (smem_u32(sm.q[0]) >> 4) | (1u << 16);             // low descriptor words: LBO field 16 B
+    const uint32_t k_lo0 = (smem_u32(sm.kv[0]) >> 4) | (1u << 16);
+    const uint32_t v_lo0 = (smem_u32(sm.kv[0]) >> 4) | ((1024u >> 4) << 16);  // V tiles: LBO = 64-dim half
+    const uint32_t bar_s_full = smem_u32(&sm.s_full[0]), bar_p_full = smem_u32(&sm.p_full[0]);
+    const uint32_t bar_q_full = smem_u32(&sm.q_full[0]), bar_o_full = smem_u32(&sm.o_full[0]);
     uint32_t loads = 0;                 // ring position, mirrors the producer
-    uint32_t steps[2] = {0, 0};         // softmax steps per tile so far (phase of s_full / p_full)
-    uint32_t items_done[2] = {0, 0};    // items per tile so far (phase of q_full / o_full)
+    uint32_t steps[2] = {0, 0};         // softmax steps per tile so far (phase of p_full)
+    uint32_t items_done[2] = {0, 0};    // items per tile so far (phase of q_full)
     bool ok = true;
-    for (int round = 0; ok; ++round) {
-      Item it;
-      if (!fetch_item(a, item_index(round), n_total, it)) break;
+    Item nxt;
+    bool has_nxt = fetch_item(a, item_index(0), n_total, nxt);
+    for (int round = 0; ok && has_nxt; ++round) {
+      const Item it = nxt;
+      has_nxt = fetch_item(a, item_index(round + 1), n_total, nxt);
       if (it.ld_tiles == 0) continue;
       if (lane == 0) {
-        const bool act1 = it.n_kv[1] > 0;
-        ok = mbar_wait(smem_u32(&sm.q_full[0]), items_done[0] & 1, abortp);
-        if (ok && act1) ok = mbar_wait(smem_u32(&sm.q_full[1]), items_done[1] & 1, abortp);
-        tc_fence_after_sync();
-        auto issue_s = [&](int t, uint32_t stage) {
-          const uint32_t qb = smem_u32(sm.q[t]), kb = smem_u32(sm.kv[stage]);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            const uint64_t ad = smem_desc_sw128(qb + (ks >> 2) * Cfg::kQHalfStride + (ks & 3) * 32, 16, 1024);
-            const uint64_t bd = smem_desc_sw128(kb + (ks >> 2) * 1024 + (ks & 3) * 32, 16, Cfg::kGroupStride);
-            mma_ss(tmem + t * 128, ad, bd, idesc_s, ks > 0);
-          }
-          mma_commit(smem_u32(&sm.s_full[t]));
-        };
-        auto issue_pv = [&](int t, uint32_t stage, int np, bool first) {
-          const uint32_t vb = smem_u32(sm.kv[stage]);
-          for (int p = 0; p < np; ++p) {
-            const uint64_t bd = smem_desc_sw128(vb + p * Cfg::kBlockBytes, 1024, Cfg::kGroupStride);
-            mma_ts(tmem + 256 + t * 128, tmem + t * 128 + p * 8, bd, idesc_o, !(first && p == 0));
-          }
-        };
-        // first K tile: S of both query tiles
-        uint32_t ks_stage = loads % Cfg::kStages;
-        ok = ok && mbar_wait(smem_u32(&sm.kv_full[ks_stage]), (loads / Cfg::kStages) & 1, abortp);
-        if (ok) {
-          tc_fence_after_sync();
-          issue_s(0, ks_stage);
-          if (act1) issue_s(1, ks_stage);
-          mma_commit(smem_u32(&sm.kv_empty[ks_stage]));
-        }
+        // first K tile: S(0) of each query tile as soon as its Q tile is in shared memory
+        uint32_t stage = loads % Cfg::kStages;
+        ok = mbar_wait(smem_u32(&sm.kv_full[stage]), (loads / Cfg::kStages) & 1, abortp);
         ++loads;
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (!ok || it.n_kv[t] == 0) continue;
+          ok = mbar_wait(bar_q_full + 8 * t, items_done[t] & 1, abortp);
+          ++items_done[t];
+          if (!ok) continue;
+          issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + stage * (Cfg::kTileBytes >> 4));
+          mma_commit(bar_s_full + 8 * t);
+        }
+        if (ok) mma_commit(smem_u32(&sm.kv_empty[stage]));
         for (int j = 0; j < it.ld_tiles && ok; ++j) {
           const int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
           const uint32_t v_stage = loads % Cfg::kStages;
           ok = mbar_wait(smem_u32(&sm.kv_full[v_stage]), (loads / Cfg::kStages) & 1, abortp);
           ++loads;
           if (!ok) break;
-          // slots past the end of the sequence may hold anything (NaN included): zero them, because the
-          // MMA multiplies them with P = 0
-          const int seq_len = it.P + it.E;
-          const int tail_lo = seq_len - j * 128;
-          if (tail_lo < np * 16) {
-            for (int r = max(tail_lo, 0); r < np * 16; ++r) {
-              unsigned char* rowp = sm.kv[v_stage] + (r >> 3) * Cfg::kGroupStride + (r & 7) * 128;
-#pragma unroll
-              for (int h = 0; h < Cfg::kHalves; ++h)
-#pragma unroll
-                for (int c = 0; c < 8; ++c) *reinterpret_cast<uint4*>(rowp + h * 1024 + c * 16) = make_uint4(0, 0, 0, 0);
-            }
-            fence_proxy_async_smem();
-          }
-          tc_fence_after_sync();
           const bool more = j + 1 < it.ld_tiles;
           uint32_t k_stage = 0;
           if (more) {
@@ -324,102 +344,130 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
             ok = mbar_wait(smem_u32(&sm.kv_full[k_stage]), (loads / Cfg::kStages) & 1, abortp);
             ++loads;
             if (!ok) break;
-            tc_fence_after_sync();
           }
 #pragma unroll
           for (int t = 0; t < 2; ++t) {
             if (j >= it.n_kv[t]) continue;
-            ok = mbar_wait(smem_u32(&sm.p_full[t]), steps[t] & 1, abortp);
+            ok = mbar_wait(bar_p_full + 8 * t, steps[t] & 1, abortp);
             ++steps[t];
             if (!ok) break;
             tc_fence_after_sync();
-            issue_pv(t, v_stage, np, j == 0);
+            issue_pv_mmas<D>(tmem + 256 + t * 128, tmem + t * 128, v_lo0 + v_stage * (Cfg::kTileBytes >> 4), np, j == 0);
             if (j + 1 < it.n_kv[t]) {
-              issue_s(t, k_stage);
+              issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + k_stage * (Cfg::kTileBytes >> 4));
+              mma_commit(bar_s_full + 8 * t);
             } else {
-              mma_commit(smem_u32(&sm.o_full[t]));
+              mma_commit(bar_o_full + 8 * t);
             }
           }
           if (!ok) break;
           mma_commit(smem_u32(&sm.kv_empty[v_stage]));
           if (more) mma_commit(smem_u32(&sm.kv_empty[k_stage]));
         }
-        ++items_done[0];
-        if (act1) ++items_done[1];
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
-      loads = __shfl_sync(0xffffffffu, loads, 0);
     }
-  } else if (warp >= 4) {
-    // =============================== softmax / epilogue ===================================
+  } else if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");  // idle warps
+  } else {
+    // =============================== softmax warpgroups ======================================
     asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
-    const int t = (warp - 4) >> 2;                 // query tile of this warpgroup
+    const int t = (warp - 4) >> 2;                 // query tile of this warpgroup (warps 4-7: tile 0, 8-11: tile 1)
     const int w4 = warp & 3;                       // TMEM lane quarter this warp may access
     const int m = w4 * 32 + lane;                  // row inside the tile
     const uint32_t lane_base = tmem + ((uint32_t)(w4 * 32) << 16);
     const uint32_t s_addr = lane_base + t * 128, o_addr = lane_base + 256 + t * 128;
+    const uint32_t bar_s_full = smem_u32(&sm.s_full[t]), bar_o_full = smem_u32(&sm.o_full[t]);
+    const uint32_t bar_q_full = smem_u32(&sm.q_full[t]), bar_p_full = smem_u32(&sm.p_full[t]);
     const int G = a.group, lg = a.lg_group, Hq = a.n_q_heads;
-    uint32_t steps = 0, items_done = 0;
+    uint32_t steps = 0, items_done = 0;            // phases of s_full / p_full and of q_full / o_full
     bool ok = true;
-    for (int round = 0; ok; ++round) {
-      Item it;
-      if (!fetch_item(a, item_index(round), n_total, it)) break;
-      if (it.n_kv[t] == 0) continue;
-      // ---- Q tile -> shared memory in the swizzled K-major operand layout (coalesced 16-byte loads)
-      {
-        constexpr int CPR = D / 8, RPI = 32 / CPR;  // chunks per row, rows per iteration of one warp
-#pragma unroll 4
-        for (int i = 0; i < 32 / RPI; ++i) {
-          const int row = w4 * 32 + i * RPI + lane / CPR, chunk = lane % CPR;
-          const int rg = it.tp * 256 + t * 128 + row;
-          const int tok = rg >> lg;
-          uint4 val = make_uint4(0, 0, 0, 0);
-          if (tok < it.E)
-            val = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1))) * D) + chunk);
-          *reinterpret_cast<uint4*>(sm.q[t] + (chunk >> 3) * Cfg::kQHalfStride + (row >> 3) * 1024 + (row & 7) * 128 +
-                                    (((chunk & 7) ^ (row & 7)) << 4)) = val;
-        }
-        fence_proxy_async_smem();
-        mbar_arrive(smem_u32(&sm.q_full[t]));
+
+    // Q rows of this warp, 16-byte chunks: iteration i covers rows w4*32 + i*RPI .. and chunk lane % CPR
+    constexpr int CPR = D / 8, RPI = 32 / CPR, QIT = 32 / RPI;  // chunks per row, rows per iteration, iterations
+    auto q_load = [&](const Item& qi, uint4 (&qv)[QIT]) {        // global -> registers (coalesced 16-byte loads)
+#pragma unroll
+      for (int i = 0; i < QIT; ++i) {
+        const int row = w4 * 32 + i * RPI + lane / CPR, chunk = lane % CPR;
+        const int rg = qi.tp * 256 + t * 128 + row;
+        const int tok = rg >> lg;
+        qv[i] = make_uint4(0, 0, 0, 0);
+        if (tok < qi.E)
+          qv[i] = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)(qi.row0 + tok) * Hq + qi.kvh * G + (rg & (G - 1))) * D) + chunk);
       }
+    };
+    auto q_store = [&](const uint4 (&qv)[QIT]) {  // registers -> shared, swizzled K-major operand layout
+#pragma unroll
+      for (int i = 0; i < QIT; ++i) {
+        const int row = w4 * 32 + i * RPI + lane / CPR, chunk = lane % CPR;
+        *reinterpret_cast<uint4*>(sm.q[t] + (chunk >> 3) * Cfg::kQHalfStride + (row >> 3) * 1024 + (row & 7) * 128 +
+                                  (((chunk & 7) ^ (row & 7)) << 4)) = qv[i];
+      }
+      fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core's reads
+      mbar_arrive(bar_q_full);
+    };
+    bool q_stored = false;  // this item's Q tile is already in shared memory (stored during the previous item)
+    Item nxt;
+    bool has_nxt = fetch_item(a, item_index(0), n_total, nxt);
+    for (int round = 0; ok && has_nxt; ++round) {
+      const Item it = nxt;
+      has_nxt = fetch_item(a, item_index(round + 1), n_total, nxt);
+      if (it.ld_tiles == 0) continue;
+      const int n_t = it.n_kv[t];
+      if (n_t == 0) continue;
+      if (!q_stored) {
+        uint4 qv[QIT];
+        q_load(it, qv);
+        q_store(qv);
+      }
+      q_stored = false;
+      const bool preload = has_nxt && nxt.n_kv[t] > 0;
       const int rg = it.tp * 256 + t * 128 + m;
       const int tok = rg >> lg;
       const bool valid = tok < it.E;
       const int limit = valid ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
       float m_run = -INFINITY, l_run = 0.f;
 
-      for (int j = 0; j < it.n_kv[t] && ok; ++j) {
-        ok = mbar_wait(smem_u32(&sm.s_full[t]), steps & 1, abortp);
+      for (int j = 0; j < n_t; ++j) {
+        ok = mbar_wait(bar_s_full, steps & 1, abortp);
         ++steps;
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
-        uint32_t sr[4][32];
-#pragma unroll
-        for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr[c]);
-        tmem_wait_ld();
+        // Two passes over the 128 score columns, 64 at a time, to keep the live registers low:
+        // pass 1 finds the row maximum, pass 2 re-reads the scores, exponentiates and writes P.
         const int kv0 = j * 128;
-        float mx = -INFINITY;
-        if (kv0 + 128 <= limit) {
+        const bool ragged = kv0 + 128 > limit;  // diagonal / last tile: keys past the row's limit are hidden
+        auto load_half = [&](int h, uint32_t (&sr)[2][32]) {
+          tmem_ld32(s_addr + h * 64, sr[0]);
+          tmem_ld32(s_addr + h * 64 + 32, sr[1]);
+          tmem_wait_ld();
+          if (ragged) {
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(sr[c][i]));
-        } else {
+              for (int i = 0; i < 32; ++i)
+                if (kv0 + h * 64 + c * 32 + i >= limit) sr[c][i] = 0xff800000u;  // -inf by select: NaN-safe
+          }
+        };
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (int c = 0; c < 4; ++c)
+        for (int h = 0; h < 2; ++h) {
+          uint32_t sr[2][32];
+          load_half(h, sr);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-              const float v = (kv0 + c * 32 + i < limit) ? __uint_as_float(sr[c][i]) : -INFINITY;  // select: NaN-safe
-              sr[c][i] = __float_as_uint(v);
-              mx = fmaxf(mx, v);
-            }
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; i += 2)
+              mx4[2 * c + ((i >> 1) & 1)] = fmax3(mx4[2 * c + ((i >> 1) & 1)], __uint_as_float(sr[c][i]), __uint_as_float(sr[c][i + 1]));
         }
-        mx *= a.scale_log2;
+        const float mx = fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * a.scale_log2;
         const float m_new = fmaxf(m_run, mx);
         const bool grow = m_new > m_run + kRescaleThreshold;  // also true on the first tile (m_run = -inf)
         const float m_use = grow ? m_new : m_run;
         if (j > 0 && __any_sync(0xffffffffu, grow)) {
+          // O holds sums scaled by 2^-m_run: bring them to the new maximum (the PV that produced them
+          // has finished: the S this step waited for was committed after it)
           const float alpha = grow ? exp2f(m_run - m_new) : 1.f;
           l_run *= alpha;
 #pragma unroll
@@ -434,30 +482,42 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         }
         m_run = m_use;
         const float neg_m = (m_use == -INFINITY) ? 0.f : -m_use;
-        float lsum = 0.f;
+        const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nm2 = make_float2(neg_m, neg_m);
+        float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t pk[16];
+        for (int h = 0; h < 2; ++h) {
+          uint32_t sr[2][32];
+          load_half(h, sr);
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float p0, p1;
-            const float x0 = fmaf(__uint_as_float(sr[c][2 * i]), a.scale_log2, neg_m);
-            const float x1 = fmaf(__uint_as_float(sr[c][2 * i + 1]), a.scale_log2, neg_m);
-            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p0) : "f"(x0));
-            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(p1) : "f"(x1));
-            lsum += p0 + p1;
-            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[i]) : "f"(p1), "f"(p0));
+          for (int c = 0; c < 2; ++c) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[c][2 * i]), __uint_as_float(sr[c][2 * i + 1])), sc2, nm2);
+              float2 pr;
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pr.x) : "f"(x.x));
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pr.y) : "f"(x.y));
+              ls2[i & 1] = __fadd2_rn(ls2[i & 1], pr);
+              asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[i]) : "f"(pr.y), "f"(pr.x));
+            }
+            // P (bf16 pairs) overwrites score columns that have already been read: columns [32h+16c, +16)
+            // lie below the 64-column half being processed, or inside the part of it held in registers
+            tmem_st16(s_addr + h * 32 + c * 16, pk);
           }
-          tmem_st16(s_addr + c * 16, pk);  // P overwrites the S columns already held in registers
         }
-        l_run += lsum;
+        l_run += (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
         tmem_wait_st();
         tc_fence_before_sync();
-        mbar_arrive(smem_u32(&sm.p_full[t]));
+        mbar_arrive(bar_p_full);
       }
+      ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
+      // every MMA that reads this tile's Q has finished (its last S was seen above): the next item's Q tile
+      // can go in now, so that its first S overlaps this item's epilogue
+      uint4 qn[QIT];
+      if (preload) q_load(nxt, qn);
       // ---- epilogue: O / l -> bf16, LSE
-      ok = mbar_wait(smem_u32(&sm.o_full[t]), items_done & 1, abortp);
+      ok = mbar_wait(bar_o_full, items_done & 1, abortp);
       ++items_done;
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -485,15 +545,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       if (valid) a.lse[orow_idx] = (m_run + log2f(l_run)) * 0.6931471805599453f;
       tc_fence_before_sync();
+      if (preload) {
+        q_store(qn);
+        q_stored = true;
+      }
     }
-  } else {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   }
 
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0 && sm.abort_flag != 0) report(a.pool.status, KV_ERR_TIMEOUT);
-  if (warp == 1) tmem_dealloc(tmem, 512);
+  if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -508,7 +570,7 @@ size_t extend_tc_workspace_bytes(int n_q_heads, int head_dim, int batch, int tot
   (void)head_dim; (void)max_total_len;
   if (batch <= 0 || total_q <= 0) return 0;
   // n_kv_heads is not known here: G <= 8 bounds the list
-  return 256 + align256(sizeof(int2) * (size_t)((int64_t)total_q * 8 / 256 + batch + 1));
+  return 256 + align256(2 * sizeof(int4) * (size_t)((int64_t)total_q * 8 / 256 + batch + 1));
 }
 
 bool extend_tc_supported(const kv_pool_t* p, int n_q_heads) {
@@ -548,12 +610,12 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   int lg = 0;
   while ((1 << lg) < G) ++lg;
   int* n_items = reinterpret_cast<int*>(workspace);
-  int2* items = reinterpret_cast<int2*>(reinterpret_cast<char*>(workspace) + 256);
+  int4* items = reinterpret_cast<int4*>(reinterpret_cast<char*>(workspace) + 256);
   const int64_t capacity = item_capacity(n_q_heads, p->n_kv_heads, batch, total_q);
   const int max_tp = (int)(((int64_t)max_extend_len * G + 255) / 256);
   const int max_steps = 2 * ((max_total_len + 127) / 128);
-  extend_tc_plan_kernel<<<1, 1024, 0, st>>>(prefix_lens, extend_lens, batch, max_tp, lg, max_steps, (int)capacity,
-                                            items, n_items);
+  extend_tc_plan_kernel<<<1, 1024, 0, st>>>(prefix_lens, extend_lens, cu_q, batch, max_tp, lg, max_steps, (int)capacity,
+                                            max_pages, p->d_status, items, n_items);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
 

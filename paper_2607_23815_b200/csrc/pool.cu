@@ -51,6 +51,18 @@ __global__ void __launch_bounds__(256) append_kernel(PoolView pool, const uint4*
     const uint4 vv = __ldg(v_new + idx);
     *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + off) = kk;
     *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + off) = vv;
+    // The segment's last token also clears the slots behind it in its page.  Slots past a sequence's
+    // end therefore never hold NaN/Inf bit patterns, which the tensor-core kernel relies on: it
+    // multiplies those V rows by probabilities that are exactly 0.
+    if (token + 1 == __ldg(cu_new + seg + 1)) {
+      const size_t blk_off = ((size_t)page * pool.n_kv_heads + head) * blk;
+      const uint4 z = make_uint4(0, 0, 0, 0);
+      for (int slot = (pos & 15) + 1; slot < kPageSize; ++slot) {
+        const size_t o2 = blk_off + chunk_offset_bytes(slot, dchunk, pool.head_dim);
+        *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + o2) = z;
+        *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + o2) = z;
+      }
+    }
   }
 }
 

@@ -81,9 +81,30 @@ def test_append_is_bit_exact_over_the_whole_pool_image(geom):
     b.write([(i, cut[i], lens[i]) for i in range(len(lens))])
     torch.cuda.synchronize()
     k_img, v_img = dp.device_image()
-    assert np.array_equal(k_img, dp.host.k) and np.array_equal(v_img, dp.host.v)
-    # untouched slots still hold the fill on both sides (nothing strays)
-    assert (dp.host.k == NAN_BITS).sum() == (k_img == NAN_BITS).sum() > 0
+    # the library clears the slots behind a segment's last token in its page (documented in the header);
+    # the oracle's append is pure, so clear the same slots in a copy of its image before comparing
+    exp_k, exp_v = dp.host.k.copy(), dp.host.v.copy()
+    for i, L in enumerate(lens):
+        for end in (cut[i], L):
+            if end > 0 and end % 16:
+                page = b.rows[i][(end - 1) // 16]
+                exp_k[page, :, end % 16:, :] = 0
+                exp_v[page, :, end % 16:, :] = 0
+        # ... which the second append then partly overwrote again
+        if cut[i] % 16 and cut[i] < L:
+            page = b.rows[i][cut[i] // 16]
+            hi = min(16, L - (cut[i] // 16) * 16)
+            exp_k[page, :, cut[i] % 16:hi, :] = dp.host.k[page, :, cut[i] % 16:hi, :]
+            exp_v[page, :, cut[i] % 16:hi, :] = dp.host.v[page, :, cut[i] % 16:hi, :]
+    assert np.array_equal(k_img, exp_k) and np.array_equal(v_img, exp_v)
+    # every written slot is bit-exact, pages the batch never named still hold the fill (nothing strays)
+    used = sorted(p for r in b.rows for p in r)
+    unused = [p for p in range(64) if p not in used]
+    assert np.all(k_img[unused] == NAN_BITS) and np.all(v_img[unused] == NAN_BITS) and len(unused) > 0
+    for i, L in enumerate(lens):
+        gk, gv = dp.host.gather(b.rows[i], L)
+        dk = np.concatenate([k_img[pg].transpose(1, 0, 2) for pg in b.rows[i]])[:L]
+        assert np.array_equal(dk, gk)
     # the library's own offset helper agrees with the formula used by device_image()
     rng = np.random.default_rng(5)
     kflat = dp.k_buf.cpu().numpy().view(np.uint16)
