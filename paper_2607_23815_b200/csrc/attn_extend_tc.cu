@@ -316,7 +316,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       const Item it = nxt;
       has_nxt = fetch_item(a, item_index(round + 1), n_total, nxt);
       if (it.ld_tiles == 0) continue;
-      if (lane == 0) {
+      {
+        // The whole warp runs this control flow (all values are warp-uniform); one elected lane issues.
         // first K tile: S(0) of each query tile as soon as its Q tile is in shared memory
         uint32_t stage = loads % Cfg::kStages;
         ok = mbar_wait(smem_u32(&sm.kv_full[stage]), (loads / Cfg::kStages) & 1, abortp);
@@ -327,10 +328,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
           ok = mbar_wait(bar_q_full + 8 * t, items_done[t] & 1, abortp);
           ++items_done[t];
           if (!ok) continue;
-          issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + stage * (Cfg::kTileBytes >> 4));
-          mma_commit(bar_s_full + 8 * t);
+          if (elect_one_sync()) {
+            issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + stage * (Cfg::kTileBytes >> 4));
+            mma_commit(bar_s_full + 8 * t);
+          }
+          __syncwarp();
         }
-        if (ok) mma_commit(smem_u32(&sm.kv_empty[stage]));
+        if (ok && elect_one_sync()) mma_commit(smem_u32(&sm.kv_empty[stage]));
+        __syncwarp();
         for (int j = 0; j < it.ld_tiles && ok; ++j) {
           const int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
           const uint32_t v_stage = loads % Cfg::kStages;
@@ -352,20 +357,26 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
             ++steps[t];
             if (!ok) break;
             tc_fence_after_sync();
-            issue_pv_mmas<D>(tmem + 256 + t * 128, tmem + t * 128, v_lo0 + v_stage * (Cfg::kTileBytes >> 4), np, j == 0);
-            if (j + 1 < it.n_kv[t]) {
-              issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + k_stage * (Cfg::kTileBytes >> 4));
-              mma_commit(bar_s_full + 8 * t);
-            } else {
-              mma_commit(bar_o_full + 8 * t);
+            if (elect_one_sync()) {
+              issue_pv_mmas<D>(tmem + 256 + t * 128, tmem + t * 128, v_lo0 + v_stage * (Cfg::kTileBytes >> 4), np, j == 0);
+              if (j + 1 < it.n_kv[t]) {
+                issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + k_stage * (Cfg::kTileBytes >> 4));
+                mma_commit(bar_s_full + 8 * t);
+              } else {
+                mma_commit(bar_o_full + 8 * t);
+              }
             }
+            __syncwarp();
           }
           if (!ok) break;
-          mma_commit(smem_u32(&sm.kv_empty[v_stage]));
-          if (more) mma_commit(smem_u32(&sm.kv_empty[k_stage]));
+          if (elect_one_sync()) {
+            mma_commit(smem_u32(&sm.kv_empty[v_stage]));
+            if (more) mma_commit(smem_u32(&sm.kv_empty[k_stage]));
+          }
+          __syncwarp();
         }
       }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
+      ok = __all_sync(0xffffffffu, ok);
     }
   } else if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");  // idle warps
