@@ -49,45 +49,49 @@ def load_peaks():
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clocks and throttle reasons through NVML (read-only) in a thread while the timed region runs."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown"}
 
     def __init__(self, index: int):
-        self.proc = None
+        import threading
+        self.sm, self.mx, self.reasons, self.err = [], None, set(), None
+        self._stop = threading.Event()
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-        except Exception:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            visible = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = int(visible.split(",")[index]) if visible and visible.split(",")[index].isdigit() else index
+            self.nv, self.h = pynvml, pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.mx = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # noqa: BLE001
+            self.nv, self.err = None, f"NVML unavailable: {e}"
+            return
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self.sm.append(float(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM)))
+                try:
+                    mask = self.nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:  # noqa: BLE001
+                    mask = self.nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception as e:  # noqa: BLE001
+                self.err = str(e)
+                return
+            time.sleep(0.002)
 
     def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            out, _ = self.proc.communicate(timeout=5)
-        except Exception:
-            self.proc.kill()
-            out = ""
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in out.strip().splitlines():
-            f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
-                continue
-            try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        if self.nv is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": [self.err]}
+        self._stop.set()
+        self.thread.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.sm) if self.sm else None, "sm_max_mhz": self.mx,
+                "samples": len(self.sm), "reasons": sorted(self.reasons)}
 
 
 def dist_setup(n_gpus):
@@ -102,21 +106,13 @@ def dist_setup(n_gpus):
 
 
 def max_over_ranks(x: float, world: int) -> float:
-    if world == 1:
-        return x
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
+    from paper_2607_23815_b200 import ranks
+    return ranks.aggregate(x, 0.0, world)[0]
 
 
 def sum_over_ranks(x: float, world: int) -> float:
-    if world == 1:
-        return x
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device="cuda")
-    dist.all_reduce(t, op=dist.ReduceOp.SUM)
-    return float(t.item())
+    from paper_2607_23815_b200 import ranks
+    return ranks.aggregate(0.0, x, world)[1]
 
 
 def barrier(world):
@@ -134,12 +130,14 @@ class L2Flusher:
         self.buf.zero_()
 
 
-def time_steps(fn, steps, warmup, flush, world, split=None):
+def time_steps(fn, steps, warmup, flush, world, split=None, on_timed_start=None):
     """Runs warmup + steps calls of fn(); returns per-step ms (device events) and, if fn records a
     mid-step event through `split`, the ms of the part after it."""
     for _ in range(warmup):
         flush(); fn(None)
     barrier(world)
+    if on_timed_start is not None:
+        on_timed_start()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True),
            torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     for i in range(steps):
@@ -170,7 +168,7 @@ def cpu_oracle_sample(wl, n_seq, kind):
     for i, L in enumerate(lens):
         n = synth.pages_needed(L, g.page_size)
         rows.append(list(range(nxt, nxt + n))); nxt += n
-        kb, vb = wl.gather_host(s.rows[i], L)
+        kb, vb = wl.source_kv("ext" if kind == "extend" else "dec", i)   # from the input generator, not the pool
         host.append(rows[-1], 0, kb, vb)
     bt = synth.block_table(rows)
     if kind == "extend":
@@ -226,11 +224,16 @@ def run_ours(args):
             mid_event.record()
         wl.extend()
 
-    sampler = ClockSampler(dev.index or 0) if rank == 0 else None
-    l0 = kvattn.kvattn_launch_count()
-    total_ms, ext_ms = time_steps(step, args.steps, args.warmup, flush, world, split=True)
-    launches = (kvattn.kvattn_launch_count() - l0) * args.steps // (args.steps + args.warmup)
-    clocks = sampler.stop() if sampler else None
+    box = {}
+
+    def timed_start():
+        box["l0"] = kvattn.kvattn_launch_count()
+        if rank == 0:
+            box["sampler"] = ClockSampler(dev.index or 0)
+
+    total_ms, ext_ms = time_steps(step, args.steps, args.warmup, flush, world, split=True, on_timed_start=timed_start)
+    launches = kvattn.kvattn_launch_count() - box["l0"]
+    clocks = box["sampler"].stop() if "sampler" in box else None
     ms_step = max_over_ranks(statistics.mean(total_ms), world)
     flops = wl.ext.flops(g)
     all_flops = sum_over_ranks(flops, world)

@@ -103,14 +103,34 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
     if (steps > 0) atomicAdd(&hist[key_of(steps)], 1);
   }
   __syncthreads();
-  if (threadIdx.x == 0) {  // exclusive prefix, heaviest bucket first
-    int run = 0;
-    for (int k = kPlanBuckets - 1; k >= 0; --k) {
-      const int c = hist[k];
-      hist[k] = run;
-      run += c;
+  // exclusive prefix over the buckets, heaviest first: thread i owns buckets B-1-2i and B-2-2i
+  {
+    __shared__ int warp_tot[32];
+    const int b0 = kPlanBuckets - 1 - 2 * (int)threadIdx.x, b1 = b0 - 1;
+    const int c0 = hist[b0], c1 = hist[b1];
+    int incl = c0 + c1;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, off);
+      if (lane >= off) incl += v;
     }
-    *n_items = min(run, capacity);
+    if (lane == 31) warp_tot[w] = incl;
+    __syncthreads();
+    if (w == 0) {
+      int t = warp_tot[lane];
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, t, off);
+        if (lane >= off) t += v;
+      }
+      warp_tot[lane] = t;  // inclusive totals of the warps
+    }
+    __syncthreads();
+    const int base = (w > 0 ? warp_tot[w - 1] : 0) + incl - (c0 + c1);
+    hist[b0] = base;
+    hist[b1] = base + c0;
+    if (threadIdx.x == blockDim.x - 1) *n_items = min(base + c0 + c1, capacity);
   }
   __syncthreads();
   for (int64_t e = threadIdx.x; e < n; e += blockDim.x) {

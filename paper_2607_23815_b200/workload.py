@@ -12,7 +12,7 @@ from typing import List, Optional
 import numpy as np
 import torch
 
-from . import kvattn, synth
+from . import kvattn, ranks, synth
 
 
 @dataclasses.dataclass
@@ -70,7 +70,7 @@ class DeviceWorkload:
 
     def __init__(self, w: synth.Workload, device="cuda", seed_offset: int = 0, write_suffix: bool = True):
         self.w, self.geom, self.device = w, w.geom, device
-        self.seed = w.seed + 7919 * seed_offset
+        self.seed = ranks.replica_seed(w.seed, seed_offset)
         g = w.geom
         self.pool = kvattn.kv_pool_create(w.num_pages, g.page_size, g.n_kv_heads, g.head_dim)
         ids = kvattn.kv_alloc(self.pool, w.num_pages)
@@ -176,6 +176,18 @@ class DeviceWorkload:
                                 e.out, e.lse) if e else None
         da = kvattn.decode_args(d.q, d.block_tables, d.ctx_lens, d.max_ctx, d.out, d.lse) if d else None
         kvattn.attn_mixed(self.pool, self.geom.n_q_heads, self.geom.scale, ea, da, self.workspace, stream)
+
+    def source_kv(self, kind: str, i: int):
+        """K/V bits of sequence i of the extend ("ext") or decode ("dec") set, re-drawn from the input
+        generator (not read back from the pool): the oracle's inputs come from here."""
+        g, dev = self.geom, self.device
+        if kind == "ext":
+            uid, length = self.ext.uids[i], self.ext.prefix[i] + self.ext.extend[i]
+        else:
+            uid, length = self.dec.uids[i], self.dec.ctx[i]
+        k = synth.normal_bf16(self.seed, synth.TAG_K, uid, 0, length, g.n_kv_heads, g.head_dim, dev)
+        v = synth.normal_bf16(self.seed, synth.TAG_V, uid, 0, length, g.n_kv_heads, g.head_dim, dev)
+        return synth.bf16_bits(k), synth.bf16_bits(v)
 
     def gather_host(self, rows, length):
         """Contiguous K/V bits of one sequence, read back through kv_gather (for the oracle's input)."""

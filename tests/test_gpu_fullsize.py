@@ -1,0 +1,141 @@
+"""Full-size configurations in the launch configuration the benchmark times: the GPU result of the whole
+batch is checked against the oracle on a sample of sequences (the oracle's K/V come from the input
+generator, its Q from the same tensor the GPU read), and by properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import paged_attention as orc
+from paper_2607_23815_b200 import kvattn, synth
+from paper_2607_23815_b200.workload import DeviceWorkload
+from harness import O_TOL, LSE_TOL, tight_ok
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_pool(wl, kind, idx):
+    """Host pool holding just the sampled sequences, on their own pages."""
+    g = wl.geom
+    s = wl.ext if kind == "ext" else wl.dec
+    lens = [(s.prefix[i] + s.extend[i]) if kind == "ext" else s.ctx[i] for i in idx]
+    host = orc.PagePool(sum(synth.pages_needed(L, 16) for L in lens), 16, g.n_kv_heads, g.head_dim)
+    rows, nxt = [], 0
+    for i, L in zip(idx, lens):
+        n = synth.pages_needed(L, 16)
+        rows.append(list(range(nxt, nxt + n))); nxt += n
+        kb, vb = wl.source_kv(kind, i)
+        host.append(rows[-1], 0, kb, vb)
+        # the pool really holds these bits where the block table says (append at full size, bit-exact)
+        gk, gv = wl.gather_host(s.rows[i], L)
+        assert np.array_equal(gk, kb) and np.array_equal(gv, vb)
+    return host, rows, lens
+
+
+def _check_extend(wl, idx):
+    g, e = wl.geom, wl.ext
+    host, rows, _ = _oracle_pool(wl, "ext", idx)
+    cu_all = e.cu_q.cpu().numpy()
+    worst = [0.0, 0.0, 0.0]
+    for k, i in enumerate(idx):
+        r0, r1 = int(cu_all[i]), int(cu_all[i + 1])
+        qb = synth.bf16_bits(e.q[r0:r1])
+        o, l = orc.attn_extend(host, qb, g.n_q_heads, [0, r1 - r0], synth.block_table([rows[k]]), [e.prefix[i]],
+                               [e.extend[i]], g.scale)
+        og, lg = e.out[r0:r1].float().cpu().numpy().astype(np.float64), e.lse[r0:r1].cpu().numpy().astype(np.float64)
+        worst = [max(worst[0], float(np.max(np.abs(og - o)))), max(worst[1], float(np.max(np.abs(lg - l)))),
+                 max(worst[2], tight_ok(og, o))]
+    assert worst[0] <= O_TOL and worst[1] <= LSE_TOL and worst[2] <= 1.0, worst
+    return worst
+
+
+def _check_decode(wl, idx):
+    g, d = wl.geom, wl.dec
+    host, rows, lens = _oracle_pool(wl, "dec", idx)
+    qb = synth.bf16_bits(d.q[idx])
+    o, l = orc.attn_decode(host, qb, g.n_q_heads, synth.block_table(rows), lens, g.scale)
+    og, lg = d.out[idx].float().cpu().numpy().astype(np.float64), d.lse[idx].cpu().numpy().astype(np.float64)
+    assert np.max(np.abs(og - o)) <= O_TOL and np.max(np.abs(lg - l)) <= LSE_TOL and tight_ok(og, o) <= 1.0
+
+
+def _any_size_properties(out, lse):
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+
+
+def _sample(lengths, k):
+    order = np.argsort(lengths)
+    pick = {int(order[0]), int(order[-1]), int(order[len(order) // 2])}
+    rng = np.random.default_rng(len(lengths))
+    while len(pick) < min(k, len(lengths)):
+        pick.add(int(rng.integers(0, len(lengths))))
+    return sorted(pick)
+
+
+def test_extend_8b_full_size():
+    wl = DeviceWorkload(synth.WORKLOADS["extend_8b"])
+    wl.extend(); torch.cuda.synchronize()
+    _any_size_properties(wl.ext.out, wl.ext.lse)
+    first = (wl.ext.out.clone(), wl.ext.lse.clone())
+    wl.extend(); torch.cuda.synchronize()                                   # run-to-run bit determinism
+    assert torch.equal(first[0].view(torch.int16), wl.ext.out.view(torch.int16)) and torch.equal(first[1], wl.ext.lse)
+    _check_extend(wl, _sample([p + e for p, e in zip(wl.ext.prefix, wl.ext.extend)], 6))
+    assert kvattn.kv_last_async_status(wl.pool) == kvattn.KV_OK
+    wl.close()
+
+
+def test_decode_8b_full_size():
+    wl = DeviceWorkload(synth.WORKLOADS["decode_8b"])
+    wl.decode(); torch.cuda.synchronize()
+    _any_size_properties(wl.dec.out, wl.dec.lse)
+    # LSE of N(0,1) scores over C keys is close to ln C + 1/2: a cheap whole-batch sanity bound
+    ctx = torch.tensor(wl.dec.ctx, device="cuda", dtype=torch.float32)
+    assert (wl.dec.lse - (torch.log(ctx) + 0.5)[:, None]).abs().max() < 0.5
+    _check_decode(wl, _sample(wl.dec.ctx, 16))
+    assert kvattn.kv_last_async_status(wl.pool) == kvattn.KV_OK
+    wl.close()
+
+
+def test_pipeline_step_full_size_mixed():
+    wl = DeviceWorkload(synth.WORKLOADS["pipeline_step"])
+    wl.mixed(); torch.cuda.synchronize()
+    _any_size_properties(wl.ext.out, wl.ext.lse); _any_size_properties(wl.dec.out, wl.dec.lse)
+    mixed = (wl.ext.out.clone(), wl.dec.out.clone())
+    wl.extend(); wl.decode(); torch.cuda.synchronize()                      # the same work, one kind at a time
+    assert torch.equal(mixed[0].view(torch.int16), wl.ext.out.view(torch.int16))
+    assert torch.equal(mixed[1].view(torch.int16), wl.dec.out.view(torch.int16))
+    _check_extend(wl, _sample([p + e for p, e in zip(wl.ext.prefix, wl.ext.extend)], 4))
+    _check_decode(wl, _sample(wl.dec.ctx, 8))
+    wl.close()
+
+
+def test_long_document_reuse_vs_from_scratch():
+    # 70B-shaped long-document reuse: the full batch runs on the GPU; the oracle checks two sampled tuples, and
+    # for the shortest tuple the GPU also recomputes prefix+suffix from scratch on fresh pages: its last E rows
+    # must agree with the reuse run (the paper's invariant) within the tolerance.
+    w = synth.WORKLOADS["long_doc_70b"]
+    wl = DeviceWorkload(w)
+    wl.extend(); torch.cuda.synchronize()
+    _any_size_properties(wl.ext.out, wl.ext.lse)
+    e, g = wl.ext, wl.geom
+    lens = [p + x for p, x in zip(e.prefix, e.extend)]
+    i = int(np.argmin(lens))
+    _check_extend(wl, [i])
+    # from-scratch prefill of the same tuple on fresh pages
+    L, P, E = lens[i], e.prefix[i], e.extend[i]
+    pages = kvattn.kv_alloc(wl.pool, synth.pages_needed(L, 16))
+    bt = torch.tensor([pages], dtype=torch.int32, device="cuda")
+    k = synth.normal_bf16(wl.seed, synth.TAG_K, e.uids[i], 0, L, g.n_kv_heads, g.head_dim, "cuda")
+    v = synth.normal_bf16(wl.seed, synth.TAG_V, e.uids[i], 0, L, g.n_kv_heads, g.head_dim, "cuda")
+    q = synth.normal_bf16(wl.seed, synth.TAG_Q, e.uids[i], 0, L, g.n_q_heads, g.head_dim, "cuda")
+    t = lambda x: torch.tensor(x, dtype=torch.int32, device="cuda")
+    kvattn.kv_append(wl.pool, k, v, t([0, L]), t([0]), None, bt)
+    out, lse = torch.empty_like(q), torch.empty((L, g.n_q_heads), device="cuda")
+    ws = torch.empty(kvattn.attn_workspace_bytes(wl.pool, g.n_q_heads, 1, L, L, 0, 0), dtype=torch.uint8, device="cuda")
+    kvattn.attn_extend(wl.pool, q, t([0, L]), bt, t([0]), t([L]), L, L, g.scale, out, lse, ws)
+    torch.cuda.synchronize()
+    r0 = int(e.cu_q[i].item())
+    assert torch.equal(q[P:].view(torch.int16), e.q[r0:r0 + E].view(torch.int16))      # same queries
+    d_o = (out[P:].float() - e.out[r0:r0 + E].float()).abs().max().item()
+    d_l = (lse[P:] - e.lse[r0:r0 + E]).abs().max().item()
+    assert d_o <= O_TOL and d_l <= LSE_TOL, (d_o, d_l)
+    assert kvattn.kv_last_async_status(wl.pool) == kvattn.KV_OK
+    wl.close()
