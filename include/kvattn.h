@@ -152,6 +152,25 @@ kv_status_t attn_decode(kv_pool_t* pool, const void* q, int n_q_heads, const int
                         const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* (No counterpart in the paper: an addition for callers that must not allocate.)
+ * Same result as attn_decode, but without a workspace argument: the split-KV scratch lives in a fixed array
+ * inside the library (attn_decode_static_scratch_bytes() = 8 MiB, resident on every GPU that loads the library
+ * until the process exits).  Meant for code that runs where device allocation is forbidden or unavailable - a
+ * plugin that was handed fixed buffers, a memory-planned or captured region of a framework, a service whose
+ * allocator is frozen after start-up - and that therefore cannot size and allocate attn_decode's workspace.
+ * The call itself performs no cudaMalloc/cudaFree and calls no allocating routine.
+ *  - Limit: a batch whose scratch need (the same formula attn_workspace_bytes() uses for decode; 0 when
+ *    max_ctx_len <= 512) exceeds the array is refused with KV_ERR_WORKSPACE; nothing is launched.
+ *  - The first call on each device looks up the array's device address (one cudaGetSymbolAddress with that
+ *    device current) and caches it; make that first call before any stream capture begins.
+ *  - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing in it needs
+ *    to be zero at entry (every slot that is read is written earlier in the same call), but two calls that
+ *    overlap on the GPU (different streams, or threads using different streams) race on it: serialise them. */
+kv_status_t attn_decode_static(kv_pool_t* pool, const void* q, int n_q_heads, const int* block_tables, int max_pages,
+                               const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
+                               void* stream);
+size_t attn_decode_static_scratch_bytes(void);
+
 typedef struct {
   const void* q; const int* cu_q; const int* block_tables; int max_pages;
   const int* prefix_lens; const int* extend_lens; int batch; int total_q;

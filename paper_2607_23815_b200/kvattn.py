@@ -55,6 +55,8 @@ _SIGNATURES = {
     "attn_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I, _I]),
     "attn_extend": (_I, [_P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_decode": (_I, [_P, _P, _I, _P, _I, _P, _I, _I, _F, _P, _P, _P, _SZ, _P]),
+    "attn_decode_static": (_I, [_P, _P, _I, _P, _I, _P, _I, _I, _F, _P, _P, _P]),
+    "attn_decode_static_scratch_bytes": (_SZ, []),
     "attn_mixed": (_I, [_P, _I, _F, C.POINTER(ExtendArgs), C.POINTER(DecodeArgs), _P, _SZ, _P]),
     "kv_check_batch": (_I, [_P, _P, _I, _P, _I, _P]),
     "kv_last_async_status": (_I, [_P]),
@@ -213,6 +215,18 @@ def attn_decode(pool: Pool, q, block_tables, ctx_lens, max_ctx_len, scale, out, 
                              _dev_ptr(lse), _dev_ptr(workspace),
                              0 if workspace is None else workspace.numel() * workspace.element_size(),
                              _stream(stream)), "attn_decode")
+
+
+def attn_decode_static(pool: Pool, q, block_tables, ctx_lens, max_ctx_len, scale, out, lse, stream=None):
+    """attn_decode for callers that cannot allocate: no workspace argument, the scratch is a fixed array inside
+    the library (see the header for the limit and the sharing rules)."""
+    _check(lib().attn_decode_static(pool.handle, _dev_ptr(q), q.shape[1], _dev_ptr(block_tables),
+                                    block_tables.shape[1], _dev_ptr(ctx_lens), q.shape[0], max_ctx_len, float(scale),
+                                    _dev_ptr(out), _dev_ptr(lse), _stream(stream)), "attn_decode_static")
+
+
+def attn_decode_static_scratch_bytes() -> int:
+    return lib().attn_decode_static_scratch_bytes()
 
 
 def extend_args(q, cu_q, block_tables, prefix_lens, extend_lens, max_extend_len, max_total_len, out, lse) -> ExtendArgs:
