@@ -36,7 +36,7 @@ HEADLINE = "extend_8b"
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
 # ncu captures summarised under profiles/; None until a capture of that kernel/workload exists.
-NCU_TRAFFIC_BYTES = {"extend_8b": None, "decode_8b": None}
+NCU_TRAFFIC_BYTES = {"extend_8b": 855_000_000, "decode_8b": 2_651_000_000}  # profiles/attn_*_kernel_*.md
 
 
 def load_peaks():
@@ -381,7 +381,7 @@ def run_reference(args):
     w = synth.WORKLOADS[args.workload]
     g = w.geom
     ext, _ = synth.draw_lengths(w)
-    n_s = min(args.cpu_sample, len(ext))
+    n_s = min(args.cpu_sample, 16, len(ext))               # about a second of host work per step
     P, E = [p for p, _ in ext[:n_s]], [e for _, e in ext[:n_s]]
     pages = sum(synth.pages_needed(p + e, g.page_size) for p, e in zip(P, E))
     host = orc.PagePool(pages, g.page_size, g.n_kv_heads, g.head_dim)
