@@ -9,8 +9,9 @@
 //   warp 0      producer: per 128-token KV tile, one 1-D bulk copy per 16-token page block
 //               (the pool keeps blocks in the MMA's 128-byte-swizzle operand layout) into a ring of
 //               shared-memory stages; completion is signalled on mbarriers.
-//   warps 1, 2  MMA issuers, one per query tile: S = Q K^T and O += P V on tcgen05 with accumulators in
+//   warp 1      MMA issuer (one elected lane): S = Q K^T and O += P V on tcgen05 with accumulators in
 //               tensor memory; P is read straight from tensor memory (it overwrites S in place).
+//   warps 2, 3  idle (they give their registers to the softmax warps).
 //   warps 4-7   softmax of query tile 0: one thread per row (= TMEM lane): masks, running max and
 //   warps 8-11  sum, exp2, P as bf16 back to TMEM, lazy rescale of O, final normalise + store.
 // The two query tiles ping-pong: while one tile's softmax runs, the tensor core works on the other.
