@@ -202,6 +202,9 @@ kv_status_t kv_last_async_status(kv_pool_t* pool);
 /* Selects the extend kernel: 0 = automatic, 1 = the small-tile kernel (rows of one KV head read K/V
  * straight from HBM), 2 = the tcgen05 tensor-core kernel.  Process-wide; for tests and benchmarks. */
 kv_status_t kvattn_set_extend_impl(int impl);
+/* Tuning: inside attn_mixed (both sets present) the persistent extend kernel takes at most n SMs, so that the
+ * HBM-bound decode kernel runs beside it on the others instead of after it.  0 = no limit.  Process-wide. */
+kv_status_t kvattn_set_mixed_extend_ctas(int n);
 /* Number of kernels this library has launched since load (all pools); for benchmark accounting. */
 int64_t kvattn_launch_count(void);
 

@@ -15,9 +15,10 @@ bool extend_tc_supported(const kv_pool_t* p, int n_q_heads);
 kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
-                             void* workspace, size_t workspace_bytes, cudaStream_t st);
+                             void* workspace, size_t workspace_bytes, int cta_cap, cudaStream_t st);
 
 static std::atomic<int> g_extend_impl{0};
+static std::atomic<int> g_mixed_extend_ctas{0};  // SMs the extend kernel may take inside attn_mixed (0 = all)
 
 static bool heads_supported(const kv_pool_t* p, int n_q_heads) {
   if (n_q_heads <= 0 || n_q_heads % p->n_kv_heads != 0) return false;
@@ -46,10 +47,10 @@ size_t attn_workspace_bytes(const kv_pool_t* p, int n_q_heads, int batch_ext, in
          align256(decode_workspace_bytes(n_q_heads, p->head_dim, batch_dec, max_ctx_len)) + 256;
 }
 
-kv_status_t attn_extend(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
-                        int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
-                        int max_extend_len, int max_total_len, float scale, void* out, float* lse, void* workspace,
-                        size_t workspace_bytes, void* stream) {
+static kv_status_t extend_impl(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                               int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                               int max_extend_len, int max_total_len, float scale, void* out, float* lse,
+                               void* workspace, size_t workspace_bytes, int cta_cap, void* stream) {
   if (p == nullptr || batch < 0 || total_q < 0 || max_pages < 0 || max_extend_len < 0 || max_total_len < 0)
     return KV_ERR_INVALID;
   if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
@@ -64,11 +65,25 @@ kv_status_t attn_extend(kv_pool_t* p, const void* q, int n_q_heads, const int* c
   if (impl == 2 && !tc_ok) return KV_ERR_UNSUPPORTED;
   if (impl == 2 || (impl == 0 && tc_ok)) {
     return launch_extend_tc(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
-                            max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes,
+                            max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, cta_cap,
                             (cudaStream_t)stream);
   }
   return launch_extend_small(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch,
                              max_extend_len, max_total_len, scale, out, lse, (cudaStream_t)stream);
+}
+
+kv_status_t attn_extend(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                        int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                        int max_extend_len, int max_total_len, float scale, void* out, float* lse, void* workspace,
+                        size_t workspace_bytes, void* stream) {
+  return extend_impl(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
+                     max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, 0, stream);
+}
+
+kv_status_t kvattn_set_mixed_extend_ctas(int n) {
+  if (n < 0) return KV_ERR_INVALID;
+  g_mixed_extend_ctas.store(n);
+  return KV_OK;
 }
 
 kv_status_t attn_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
@@ -101,17 +116,18 @@ kv_status_t attn_mixed(kv_pool_t* p, int n_q_heads, float scale, const attn_exte
   if (ext_bytes > workspace_bytes) return KV_ERR_WORKSPACE;
   char* ws = reinterpret_cast<char*>(workspace);
   if (has_ext && has_dec) {
-    // decode (HBM-bound) goes to the pool's side stream, extend (tensor-bound) stays on the caller's
+    // The persistent extend kernel (tensor-bound) goes first on the caller's stream and may be limited to a
+    // part of the SMs; decode (HBM-bound) follows on the pool's side stream and fills the others.
     KV_CUDA_OK(cudaEventRecord(p->ev_fork, st));
     KV_CUDA_OK(cudaStreamWaitEvent(p->side_stream, p->ev_fork, 0));
-    kv_status_t s = attn_decode(p, dec->q, n_q_heads, dec->block_tables, dec->max_pages, dec->ctx_lens, dec->batch,
-                                dec->max_ctx_len, scale, dec->out, dec->lse, ws ? ws + ext_bytes : nullptr,
-                                workspace_bytes - ext_bytes, p->side_stream);
+    kv_status_t s = extend_impl(p, ext->q, n_q_heads, ext->cu_q, ext->block_tables, ext->max_pages, ext->prefix_lens,
+                                ext->extend_lens, ext->batch, ext->total_q, ext->max_extend_len, ext->max_total_len,
+                                scale, ext->out, ext->lse, ws, ext_bytes, g_mixed_extend_ctas.load(), st);
     kv_status_t s2 = KV_OK;
     if (s == KV_OK)
-      s2 = attn_extend(p, ext->q, n_q_heads, ext->cu_q, ext->block_tables, ext->max_pages, ext->prefix_lens,
-                       ext->extend_lens, ext->batch, ext->total_q, ext->max_extend_len, ext->max_total_len, scale,
-                       ext->out, ext->lse, ws, ext_bytes, st);
+      s2 = attn_decode(p, dec->q, n_q_heads, dec->block_tables, dec->max_pages, dec->ctx_lens, dec->batch,
+                       dec->max_ctx_len, scale, dec->out, dec->lse, ws ? ws + ext_bytes : nullptr,
+                       workspace_bytes - ext_bytes, p->side_stream);
     // always rejoin, so that the caller's stream stays ordered after whatever was launched
     KV_CUDA_OK(cudaEventRecord(p->ev_join, p->side_stream));
     KV_CUDA_OK(cudaStreamWaitEvent(st, p->ev_join, 0));

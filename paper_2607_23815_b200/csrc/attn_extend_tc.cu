@@ -461,11 +461,21 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       float m_run = -INFINITY, l_run = 0.f;
 
       for (int j = 0; j < n_t; ++j) {
+        // The next item's Q rows are fetched while this thread waits for the item's last S; once that S is
+        // there, every MMA that reads this tile's Q buffer has finished and the buffer can be refilled, so the
+        // next item's first S overlaps this item's last softmax step and epilogue.
+        const bool refill = preload && j + 1 == n_t;
+        uint4 qn[QIT];
+        if (refill) q_load(nxt, qn);
         ok = mbar_wait(bar_s_full, steps & 1, abortp);
         ++steps;
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
+        if (refill) {
+          q_store(qn);
+          q_stored = true;
+        }
         // Two passes over the 128 score columns, 64 at a time, to keep the live registers low:
         // pass 1 finds the row maximum, pass 2 re-reads the scores, exponentiates and writes P.
         const int kv0 = j * 128;
@@ -544,10 +554,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      // every MMA that reads this tile's Q has finished (its last S was seen above): the next item's Q tile
-      // can go in now, so that its first S overlaps this item's epilogue
-      uint4 qn[QIT];
-      if (preload) q_load(nxt, qn);
       // ---- epilogue: O / l -> bf16, LSE
       ok = mbar_wait(bar_o_full, items_done & 1, abortp);
       ++items_done;
@@ -577,10 +583,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       if (valid) a.lse[orow_idx] = (m_run + log2f(l_run)) * 0.6931471805599453f;
       tc_fence_before_sync();
-      if (preload) {
-        q_store(qn);
-        q_stored = true;
-      }
     }
   }
 
@@ -612,7 +614,7 @@ bool extend_tc_supported(const kv_pool_t* p, int n_q_heads) {
 }
 
 template <int D>
-static kv_status_t launch_tc(const TcArgs& a, int n_items_bound, cudaStream_t st) {
+static kv_status_t launch_tc(const TcArgs& a, int n_items_bound, int cta_cap, cudaStream_t st) {
   static int sm_count = 0;
   if (sm_count == 0) {
     int dev = 0;
@@ -625,7 +627,8 @@ static kv_status_t launch_tc(const TcArgs& a, int n_items_bound, cudaStream_t st
     KV_CUDA_OK(cudaFuncSetAttribute(attn_extend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = true;
   }
-  const int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
+  int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
+  if (cta_cap > 0 && grid > cta_cap) grid = cta_cap;  // leave the other SMs to work that runs beside this kernel
   attn_extend_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(a);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
@@ -635,7 +638,7 @@ static kv_status_t launch_tc(const TcArgs& a, int n_items_bound, cudaStream_t st
 kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
-                             void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                             void* workspace, size_t workspace_bytes, int cta_cap, cudaStream_t st) {
   const size_t need = extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch, total_q, max_total_len);
   if (workspace == nullptr || workspace_bytes < need) return KV_ERR_WORKSPACE;
   const int G = n_q_heads / p->n_kv_heads;
@@ -670,8 +673,8 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   a.n_items = n_items;
   const int64_t bound = (int64_t)batch * max_tp * p->n_kv_heads;
   const int n_bound = bound > (1 << 30) ? (1 << 30) : (int)bound;
-  if (p->head_dim == 128) return launch_tc<128>(a, n_bound, st);
-  return launch_tc<64>(a, n_bound, st);
+  if (p->head_dim == 128) return launch_tc<128>(a, n_bound, cta_cap, st);
+  return launch_tc<64>(a, n_bound, cta_cap, st);
 }
 
 }  // namespace kvattn

@@ -61,6 +61,7 @@ _SIGNATURES = {
     "kv_check_batch": (_I, [_P, _P, _I, _P, _I, _P]),
     "kv_last_async_status": (_I, [_P]),
     "kvattn_set_extend_impl": (_I, [_I]),
+    "kvattn_set_mixed_extend_ctas": (_I, [_I]),
     "kvattn_launch_count": (_I64, []),
 }
 
@@ -259,6 +260,10 @@ def kv_last_async_status(pool: Pool) -> int:
 
 def kvattn_set_extend_impl(impl: int):
     _check(lib().kvattn_set_extend_impl(impl), "kvattn_set_extend_impl")
+
+
+def kvattn_set_mixed_extend_ctas(n: int):
+    _check(lib().kvattn_set_mixed_extend_ctas(n), "kvattn_set_mixed_extend_ctas")
 
 
 def kvattn_launch_count() -> int:
