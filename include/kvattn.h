@@ -160,7 +160,7 @@ kv_status_t attn_decode(kv_pool_t* pool, const void* q, int n_q_heads, const int
  * allocator is frozen after start-up - and that therefore cannot size and allocate attn_decode's workspace.
  * The call itself performs no cudaMalloc/cudaFree and calls no allocating routine.
  *  - Limit: a batch whose scratch need (the same formula attn_workspace_bytes() uses for decode; 0 when
- *    max_ctx_len <= 512) exceeds the array is refused with KV_ERR_WORKSPACE; nothing is launched.
+ *    max_ctx_len <= 1024) exceeds the array is refused with KV_ERR_WORKSPACE; nothing is launched.
  *  - The first call on each device looks up the array's device address (one cudaGetSymbolAddress with that
  *    device current) and caches it; make that first call before any stream capture begins.
  *  - All calls on a device share the one array, and it keeps the previous call's contents.  Nothing in it needs

@@ -14,7 +14,7 @@
 namespace kvattn {
 
 constexpr int kChunkPages = 32;                       // pages per batch of block-table entries (one per lane)
-constexpr int kDecodeChunkTokens = kChunkPages * 16;  // split size of decode: a function of nothing but this constant
+constexpr int kDecodeChunkTokens = kChunkPages * 16 * 2;  // split size of decode: a function of nothing but this constant
 
 struct SmallArgs {
   PoolView pool;

@@ -12,14 +12,14 @@ pytestmark = pytest.mark.gpu
 @pytest.mark.parametrize("hq,hkv,d", [(4, 2, 64), (8, 8, 64), (8, 1, 64), (32, 8, 128), (8, 2, 128), (4, 4, 128)])
 def test_decode_edge_lengths(hq, hkv, d):
     geom = synth.Geometry(hq, hkv, d)
-    lens = [1, 2, 15, 16, 17, 31, 33, 511, 512, 513, 1025, 0, 100]
-    dp = DualPool(geom, 256, seed=100 + hq + d)
+    lens = [1, 2, 15, 16, 17, 31, 33, 511, 513, 1023, 1024, 1025, 0, 100]
+    dp = DualPool(geom, 512, seed=100 + hq + d)
     b = Batch(dp, lens)
     b.write([(i, 0, L) for i, L in enumerate(lens)])
     res = run_decode(dp, b, lens)
     d_o, d_l, t = assert_close(res, f"decode {hq}/{hkv}/{d}")
     # the empty sequence: O = 0, LSE = -inf
-    assert np.all(res["o"][11] == 0) and np.all(np.isneginf(res["lse"][11]))
+    assert np.all(res["o"][12] == 0) and np.all(np.isneginf(res["lse"][12]))
     assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
     dp.close()
 

@@ -58,7 +58,7 @@ def test_static_scratch_refuses_batches_beyond_its_limit():
     dp = DualPool(geom, 512, seed=910, with_oracle=False)
     limit = kvattn.attn_decode_static_scratch_bytes()
     assert limit == 8 << 20
-    batch, max_ctx = 256, 4096                                           # needs about 33 MB of partials
+    batch, max_ctx = 256, 4096                                           # needs about 17 MB of partials
     assert kvattn.attn_workspace_bytes(dp.pool, geom.n_q_heads, 0, 0, 0, batch, max_ctx) > limit
     q = torch.zeros((batch, geom.n_q_heads, geom.head_dim), dtype=torch.bfloat16, device="cuda")
     bt = torch.zeros((batch, 256), dtype=torch.int32, device="cuda")
