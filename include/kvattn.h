@@ -61,7 +61,8 @@ typedef enum {
   KV_ERR_UNSUPPORTED = 5,   /* shape outside the supported set                                 */
   KV_ERR_CUDA = 6,          /* a CUDA runtime call failed (allocation, launch)                 */
   KV_ERR_TIMEOUT = 7,       /* a bounded device-side wait gave up                              */
-  KV_ERR_WORKSPACE = 8      /* workspace pointer NULL or smaller than attn_workspace_bytes()   */
+  KV_ERR_WORKSPACE = 8,     /* workspace pointer NULL or smaller than attn_workspace_bytes()   */
+  KV_ERR_PINNED = 9         /* kv_evict, or the last kv_free, of a page that is pinned          */
 } kv_status_t;
 
 const char* kv_status_str(kv_status_t s);
@@ -101,6 +102,29 @@ kv_status_t kv_free(kv_pool_t* pool, const int* page_ids /*host*/, int n);
  * evicted at any time").  Same as kv_free plus the eviction counter and the optional poison fill;
  * the former owner must treat its prefix as lost and re-prefill (Section 2.2). */
 kv_status_t kv_evict(kv_pool_t* pool, const int* page_ids /*host*/, int n);
+
+/* ---- sharing, pinning, eviction order (host; mutex-guarded) --------------------------------
+ * A join creates many dependent tasks over one parent tuple, whose prefix pages they all read (Section 5.1;
+ * Algorithm 1, Complete: the parent's memory is released when all its children are done): kv_ref adds an owner
+ * to allocated pages, and kv_free only returns a page to the free list when its last owner frees it.
+ * Explicit pinning (Section 6, "Explicit and virtual pinning"): a pinned block cannot be evicted until the
+ * scheduler unpins it; kv_evict / kv_evict_lru never take a pinned page (kv_evict: KV_ERR_PINNED, nothing
+ * changed), and the last owner cannot kv_free it while it is pinned either.  Pins are counted.
+ * Deadlock recovery (Section 6): when requests wait while nothing runs, the scheduler unpins everything and
+ * falls back to virtual pinning: kv_unpin_all.
+ * Eviction order: the engine evicts least-recently-used blocks (Section 2.2, Section 6).  The pool keeps a
+ * logical clock per page, set by kv_alloc and kv_touch; kv_evict_lru(n) evicts up to n unpinned allocated
+ * pages, least recently used first, whoever owns them (their owners must treat that prefix as lost), and
+ * reports which.  All calls validate first and change nothing on error (KV_ERR_NOT_ALLOCATED for a page that
+ * is not allocated, KV_ERR_INVALID for kv_unpin of a page that is not pinned).                              */
+kv_status_t kv_ref(kv_pool_t* pool, const int* page_ids /*host*/, int n);
+kv_status_t kv_pin(kv_pool_t* pool, const int* page_ids /*host*/, int n);
+kv_status_t kv_unpin(kv_pool_t* pool, const int* page_ids /*host, no repeats*/, int n);
+kv_status_t kv_unpin_all(kv_pool_t* pool, int* n_unpinned /*host, may be NULL: pages that were pinned*/);
+kv_status_t kv_touch(kv_pool_t* pool, const int* page_ids /*host*/, int n);
+kv_status_t kv_evict_lru(kv_pool_t* pool, int n, int* out_page_ids /*host [n]*/, int* n_evicted /*host*/);
+/* Test surface: state of one page (any pointer may be NULL). */
+kv_status_t kv_page_info(const kv_pool_t* pool, int page, int* allocated, int* refs, int* pins);
 
 /* ---- kv_append: materialise new tokens' K/V in their pages (Section 2.1: prefill "materializes
  *      per-layer key-value tensors") ------------------------------------------------------- */

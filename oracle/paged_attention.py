@@ -60,19 +60,32 @@ def widen(bits: np.ndarray) -> np.ndarray:
 # --------------------------------------------------------------------------- #
 # page pool (host image) and allocator
 # --------------------------------------------------------------------------- #
-class FreeList:
-    """LIFO free list over page ids 0..num_pages-1.
+class PinnedError(Exception):
+    """kv_evict, or the last kv_free, of a pinned page."""
 
-    Documented order: a fresh list hands out 0, 1, 2, ...; freed pages are
-    pushed in the order given and popped last-in-first-out.  ``alloc`` is
-    all-or-nothing.  Freeing a page that is not allocated is an error with no
-    partial effect.
+
+class FreeList:
+    """LIFO free list over page ids 0..num_pages-1, with owners, pins and an LRU clock.
+
+    Documented order: a fresh list hands out 0, 1, 2, ...; released pages are pushed in the order given and
+    popped last-in-first-out.  ``alloc`` is all-or-nothing.  Every call validates first and changes nothing
+    on error.
+
+    Sharing (paper Section 5.1; Algorithm 1, Complete: a parent's memory is released when all of its children
+    are done): ``ref`` adds an owner, ``free`` removes one, and the page goes back when the last owner frees it.
+    Explicit pinning (Section 6): a pinned page is never evicted (``evict`` raises, ``evict_lru`` skips it) and
+    its last owner cannot free it; ``unpin_all`` is the deadlock fallback.  Eviction order (Sections 2.2, 6):
+    least recently used first, by a logical clock that ``alloc`` and ``touch`` advance.
     """
 
     def __init__(self, num_pages: int):
         self.num_pages = num_pages
         self.stack = list(range(num_pages - 1, -1, -1))   # pop() gives 0 first
         self.allocated = np.zeros(num_pages, dtype=bool)
+        self.refs = [0] * num_pages
+        self.pins = [0] * num_pages
+        self.last_use = [0] * num_pages
+        self.clock = 0
         self.evicted_total = 0
 
     def alloc(self, n: int):
@@ -81,26 +94,84 @@ class FreeList:
         if n > len(self.stack):
             return None                                    # out of pages: caller defers
         ids = [self.stack.pop() for _ in range(n)]
-        self.allocated[ids] = True
+        for p in ids:
+            self.allocated[p] = True
+            self.refs[p], self.pins[p] = 1, 0
+            self.clock += 1
+            self.last_use[p] = self.clock
         return ids
 
-    def _release(self, ids):
-        ids = list(ids)
+    def _check(self, ids, unique):
         seen = set()
         for p in ids:
-            if p < 0 or p >= self.num_pages or not self.allocated[p] or p in seen:
+            if p < 0 or p >= self.num_pages or not self.allocated[p] or (unique and p in seen):
                 raise KeyError(f"page {p} is not allocated")
             seen.add(p)
-        for p in ids:
-            self.allocated[p] = False
-            self.stack.append(p)
+
+    def _drop(self, p):
+        self.allocated[p] = False
+        self.refs[p] = 0
+        self.stack.append(p)
 
     def free(self, ids):
-        self._release(ids)
+        ids = list(ids)
+        self._check(ids, unique=True)
+        if any(self.pins[p] > 0 and self.refs[p] == 1 for p in ids):
+            raise PinnedError()
+        for p in ids:
+            self.refs[p] -= 1
+            if self.refs[p] == 0:
+                self._drop(p)
 
     def evict(self, ids):
-        self._release(ids)
-        self.evicted_total += len(list(ids))
+        ids = list(ids)
+        self._check(ids, unique=True)
+        if any(self.pins[p] > 0 for p in ids):
+            raise PinnedError()
+        for p in ids:
+            self._drop(p)
+        self.evicted_total += len(ids)
+
+    def ref(self, ids):
+        ids = list(ids)
+        self._check(ids, unique=False)
+        for p in ids:
+            self.refs[p] += 1
+
+    def pin(self, ids):
+        ids = list(ids)
+        self._check(ids, unique=False)
+        for p in ids:
+            self.pins[p] += 1
+
+    def unpin(self, ids):
+        ids = list(ids)
+        self._check(ids, unique=True)
+        if any(self.pins[p] == 0 for p in ids):
+            raise ValueError("page is not pinned")
+        for p in ids:
+            self.pins[p] -= 1
+
+    def unpin_all(self) -> int:
+        n = sum(1 for c in self.pins if c > 0)
+        self.pins = [0] * self.num_pages
+        return n
+
+    def touch(self, ids):
+        ids = list(ids)
+        self._check(ids, unique=False)
+        for p in ids:
+            self.clock += 1
+            self.last_use[p] = self.clock
+
+    def evict_lru(self, n: int):
+        cand = [p for p in range(self.num_pages) if self.allocated[p] and self.pins[p] == 0]
+        cand.sort(key=lambda p: self.last_use[p])
+        out = cand[:n]
+        for p in out:
+            self._drop(p)
+        self.evicted_total += len(out)
+        return out
 
     @property
     def free_pages(self) -> int:

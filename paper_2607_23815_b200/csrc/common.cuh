@@ -59,6 +59,10 @@ struct kv_pool {
   std::vector<int> free_stack;       // back() is handed out next
   std::vector<uint8_t> allocated;    // per page
   std::vector<uint32_t> mark;        // duplicate detection in one release call
+  std::vector<uint16_t> refs;        // owners of an allocated page (kv_alloc: 1, kv_ref: +1, kv_free: -1)
+  std::vector<uint16_t> pins;        // pin count: a pinned page cannot be evicted
+  std::vector<uint64_t> last_use;    // logical clock of the last kv_alloc / kv_touch, for kv_evict_lru
+  uint64_t clock;
   uint32_t mark_epoch;
   int64_t evicted_total;
   // second stream + events used by attn_mixed to overlap the two kinds of work

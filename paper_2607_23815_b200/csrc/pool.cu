@@ -143,6 +143,7 @@ const char* kv_status_str(kv_status_t s) {
     case KV_ERR_CUDA: return "CUDA runtime error";
     case KV_ERR_TIMEOUT: return "device-side wait timed out";
     case KV_ERR_WORKSPACE: return "workspace missing or too small";
+    case KV_ERR_PINNED: return "page is pinned";
   }
   return "unknown status";
 }
@@ -180,6 +181,10 @@ static kv_status_t pool_create_impl(int num_pages, int page_size, int n_kv_heads
   p->free_stack.resize(num_pages);
   for (int i = 0; i < num_pages; ++i) p->free_stack[i] = num_pages - 1 - i;  // back() == 0 first
   p->allocated.assign(num_pages, 0);
+  p->refs.assign(num_pages, 0);
+  p->pins.assign(num_pages, 0);
+  p->last_use.assign(num_pages, 0);
+  p->clock = 0;
   p->mark.assign(num_pages, 0);
   *out = p;
   return KV_OK;
@@ -251,8 +256,36 @@ kv_status_t kv_alloc(kv_pool_t* p, int n, int* out_page_ids) {
     const int id = p->free_stack.back();
     p->free_stack.pop_back();
     p->allocated[id] = 1;
+    p->refs[id] = 1;
+    p->pins[id] = 0;
+    p->last_use[id] = ++p->clock;
     out_page_ids[i] = id;
   }
+  return KV_OK;
+}
+
+// Marks the ids of one call; returns false on an id that is out of range, not allocated or (if `unique`) repeated.
+static bool check_ids(kv_pool_t* p, const int* ids, int n, bool unique) {
+  if (++p->mark_epoch == 0) {  // epoch wrapped: clear the marks
+    std::fill(p->mark.begin(), p->mark.end(), 0u);
+    p->mark_epoch = 1;
+  }
+  for (int i = 0; i < n; ++i) {
+    const int id = ids[i];
+    if (id < 0 || id >= p->num_pages || !p->allocated[id]) return false;
+    if (unique && p->mark[id] == p->mark_epoch) return false;
+    p->mark[id] = p->mark_epoch;
+  }
+  return true;
+}
+
+static kv_status_t poison_pages(kv_pool_t* p, const int* ids, int n) {
+  if (!p->poison || n <= 0) return KV_OK;
+  KV_CUDA_OK(cudaMemcpy(p->d_scratch_ids, ids, sizeof(int) * (size_t)n, cudaMemcpyHostToDevice));
+  poison_kernel<<<n < 1184 ? n : 1184, 256>>>(p->view(), p->d_scratch_ids, n);
+  count_launch();
+  KV_CUDA_OK(cudaGetLastError());
+  KV_CUDA_OK(cudaDeviceSynchronize());
   return KV_OK;
 }
 
@@ -260,34 +293,109 @@ static kv_status_t release_pages(kv_pool_t* p, const int* ids, int n, bool evict
   if (p == nullptr || n < 0 || (n > 0 && ids == nullptr)) return KV_ERR_INVALID;
   {
     std::lock_guard<std::mutex> g(p->mu);
-    if (++p->mark_epoch == 0) {  // epoch wrapped: clear the marks
-      std::fill(p->mark.begin(), p->mark.end(), 0u);
-      p->mark_epoch = 1;
+    if (!check_ids(p, ids, n, true)) return KV_ERR_NOT_ALLOCATED;  // nothing has been changed yet
+    for (int i = 0; i < n; ++i) {
+      // a pinned page is never evicted, and its last owner cannot drop it either
+      if (p->pins[ids[i]] > 0 && (evict || p->refs[ids[i]] == 1)) return KV_ERR_PINNED;
     }
     for (int i = 0; i < n; ++i) {
       const int id = ids[i];
-      if (id < 0 || id >= p->num_pages || !p->allocated[id] || p->mark[id] == p->mark_epoch)
-        return KV_ERR_NOT_ALLOCATED;  // nothing has been changed yet
-      p->mark[id] = p->mark_epoch;
-    }
-    for (int i = 0; i < n; ++i) {
-      p->allocated[ids[i]] = 0;
-      p->free_stack.push_back(ids[i]);
+      if (!evict && --p->refs[id] > 0) continue;  // other owners remain
+      p->allocated[id] = 0;
+      p->refs[id] = 0;
+      p->free_stack.push_back(id);
     }
     if (evict) p->evicted_total += n;
   }
-  if (evict && p->poison && n > 0) {
-    KV_CUDA_OK(cudaMemcpy(p->d_scratch_ids, ids, sizeof(int) * (size_t)n, cudaMemcpyHostToDevice));
-    poison_kernel<<<n < 1184 ? n : 1184, 256>>>(p->view(), p->d_scratch_ids, n);
-    count_launch();
-    KV_CUDA_OK(cudaGetLastError());
-    KV_CUDA_OK(cudaDeviceSynchronize());
-  }
-  return KV_OK;
+  return evict ? poison_pages(p, ids, n) : KV_OK;
 }
 
 kv_status_t kv_free(kv_pool_t* p, const int* page_ids, int n) { return release_pages(p, page_ids, n, false); }
 kv_status_t kv_evict(kv_pool_t* p, const int* page_ids, int n) { return release_pages(p, page_ids, n, true); }
+
+kv_status_t kv_ref(kv_pool_t* p, const int* page_ids, int n) {
+  if (p == nullptr || n < 0 || (n > 0 && page_ids == nullptr)) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(p->mu);
+  if (!check_ids(p, page_ids, n, false)) return KV_ERR_NOT_ALLOCATED;
+  for (int i = 0; i < n; ++i)
+    if (p->refs[page_ids[i]] >= 0xFFFF) return KV_ERR_INVALID;
+  for (int i = 0; i < n; ++i) ++p->refs[page_ids[i]];
+  return KV_OK;
+}
+
+kv_status_t kv_pin(kv_pool_t* p, const int* page_ids, int n) {
+  if (p == nullptr || n < 0 || (n > 0 && page_ids == nullptr)) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(p->mu);
+  if (!check_ids(p, page_ids, n, false)) return KV_ERR_NOT_ALLOCATED;
+  for (int i = 0; i < n; ++i)
+    if (p->pins[page_ids[i]] >= 0xFFFF) return KV_ERR_INVALID;
+  for (int i = 0; i < n; ++i) ++p->pins[page_ids[i]];
+  return KV_OK;
+}
+
+kv_status_t kv_unpin(kv_pool_t* p, const int* page_ids, int n) {
+  if (p == nullptr || n < 0 || (n > 0 && page_ids == nullptr)) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(p->mu);
+  if (!check_ids(p, page_ids, n, true)) return KV_ERR_NOT_ALLOCATED;
+  for (int i = 0; i < n; ++i)
+    if (p->pins[page_ids[i]] == 0) return KV_ERR_INVALID;  // not pinned; nothing has been changed yet
+  for (int i = 0; i < n; ++i) --p->pins[page_ids[i]];
+  return KV_OK;
+}
+
+kv_status_t kv_unpin_all(kv_pool_t* p, int* n_unpinned) {
+  if (p == nullptr) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(p->mu);
+  int cnt = 0;
+  for (int id = 0; id < p->num_pages; ++id) {
+    if (p->pins[id] > 0) ++cnt;
+    p->pins[id] = 0;
+  }
+  if (n_unpinned) *n_unpinned = cnt;
+  return KV_OK;
+}
+
+kv_status_t kv_touch(kv_pool_t* p, const int* page_ids, int n) {
+  if (p == nullptr || n < 0 || (n > 0 && page_ids == nullptr)) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(p->mu);
+  if (!check_ids(p, page_ids, n, false)) return KV_ERR_NOT_ALLOCATED;
+  for (int i = 0; i < n; ++i) p->last_use[page_ids[i]] = ++p->clock;
+  return KV_OK;
+}
+
+kv_status_t kv_evict_lru(kv_pool_t* p, int n, int* out_page_ids, int* n_evicted) {
+  if (p == nullptr || n < 0 || n_evicted == nullptr || (n > 0 && out_page_ids == nullptr)) return KV_ERR_INVALID;
+  int cnt = 0;
+  {
+    std::lock_guard<std::mutex> g(p->mu);
+    std::vector<int> cand;
+    for (int id = 0; id < p->num_pages; ++id)
+      if (p->allocated[id] && p->pins[id] == 0) cand.push_back(id);
+    cnt = n < (int)cand.size() ? n : (int)cand.size();
+    // least recently used first; the clock is strictly increasing, so there are no ties
+    std::partial_sort(cand.begin(), cand.begin() + cnt, cand.end(),
+                      [&](int a, int b) { return p->last_use[a] < p->last_use[b]; });
+    for (int i = 0; i < cnt; ++i) {
+      const int id = cand[i];
+      p->allocated[id] = 0;
+      p->refs[id] = 0;
+      p->free_stack.push_back(id);
+      out_page_ids[i] = id;
+    }
+    p->evicted_total += cnt;
+  }
+  *n_evicted = cnt;
+  return poison_pages(p, out_page_ids, cnt);
+}
+
+kv_status_t kv_page_info(const kv_pool_t* p, int page, int* allocated, int* refs, int* pins) {
+  if (p == nullptr || page < 0 || page >= p->num_pages) return KV_ERR_INVALID;
+  std::lock_guard<std::mutex> g(const_cast<kv_pool_t*>(p)->mu);
+  if (allocated) *allocated = p->allocated[page];
+  if (refs) *refs = p->refs[page];
+  if (pins) *pins = p->pins[page];
+  return KV_OK;
+}
 
 kv_status_t kv_append(kv_pool_t* p, const void* k_new, const void* v_new, const int* cu_new, const int* start_pos,
                       const int* seg_row, const int* block_tables, int max_pages, int n_segments, int total_new,

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkvattn.so")
 
 KV_OK, KV_ERR_INVALID, KV_ERR_OOM, KV_ERR_NOT_ALLOCATED, KV_ERR_BOUNDS = 0, 1, 2, 3, 4
-KV_ERR_UNSUPPORTED, KV_ERR_CUDA, KV_ERR_TIMEOUT, KV_ERR_WORKSPACE = 5, 6, 7, 8
+KV_ERR_UNSUPPORTED, KV_ERR_CUDA, KV_ERR_TIMEOUT, KV_ERR_WORKSPACE, KV_ERR_PINNED = 5, 6, 7, 8, 9
 
 
 class KvError(RuntimeError):
@@ -50,6 +50,13 @@ _SIGNATURES = {
     "kv_alloc": (_I, [_P, _I, C.POINTER(_I)]),
     "kv_free": (_I, [_P, C.POINTER(_I), _I]),
     "kv_evict": (_I, [_P, C.POINTER(_I), _I]),
+    "kv_ref": (_I, [_P, C.POINTER(_I), _I]),
+    "kv_pin": (_I, [_P, C.POINTER(_I), _I]),
+    "kv_unpin": (_I, [_P, C.POINTER(_I), _I]),
+    "kv_unpin_all": (_I, [_P, C.POINTER(_I)]),
+    "kv_touch": (_I, [_P, C.POINTER(_I), _I]),
+    "kv_evict_lru": (_I, [_P, _I, C.POINTER(_I), C.POINTER(_I)]),
+    "kv_page_info": (_I, [_P, _I, C.POINTER(_I), C.POINTER(_I), C.POINTER(_I)]),
     "kv_append": (_I, [_P, _P, _P, _P, _P, _P, _P, _I, _I, _I, _P]),
     "kv_gather": (_I, [_P, _P, _I, _P, _P, _P]),
     "attn_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I, _I]),
@@ -180,6 +187,40 @@ def kv_free(pool: Pool, page_ids: Sequence[int]):
 
 def kv_evict(pool: Pool, page_ids: Sequence[int]):
     _check(lib().kv_evict(pool.handle, _int_array(page_ids), len(page_ids)), "kv_evict")
+
+
+def kv_ref(pool: Pool, page_ids: Sequence[int]):
+    _check(lib().kv_ref(pool.handle, _int_array(page_ids), len(page_ids)), "kv_ref")
+
+
+def kv_pin(pool: Pool, page_ids: Sequence[int]):
+    _check(lib().kv_pin(pool.handle, _int_array(page_ids), len(page_ids)), "kv_pin")
+
+
+def kv_unpin(pool: Pool, page_ids: Sequence[int]):
+    _check(lib().kv_unpin(pool.handle, _int_array(page_ids), len(page_ids)), "kv_unpin")
+
+
+def kv_unpin_all(pool: Pool) -> int:
+    n = C.c_int()
+    _check(lib().kv_unpin_all(pool.handle, C.byref(n)), "kv_unpin_all")
+    return n.value
+
+
+def kv_touch(pool: Pool, page_ids: Sequence[int]):
+    _check(lib().kv_touch(pool.handle, _int_array(page_ids), len(page_ids)), "kv_touch")
+
+
+def kv_evict_lru(pool: Pool, n: int):
+    out, cnt = (C.c_int * max(n, 1))(), C.c_int()
+    _check(lib().kv_evict_lru(pool.handle, n, out, C.byref(cnt)), "kv_evict_lru")
+    return list(out[:cnt.value])
+
+
+def kv_page_info(pool: Pool, page: int):
+    a, r, p = C.c_int(), C.c_int(), C.c_int()
+    _check(lib().kv_page_info(pool.handle, page, C.byref(a), C.byref(r), C.byref(p)), "kv_page_info")
+    return a.value, r.value, p.value
 
 
 def kv_append(pool: Pool, k_new, v_new, cu_new, start_pos, seg_row, block_tables, stream=None):

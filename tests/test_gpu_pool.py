@@ -164,3 +164,58 @@ def test_evict_with_poison_overwrites_the_pages():
     torch.cuda.synchronize()
     assert torch.isnan(out[16:32].float()).all() and torch.equal(out[:16], k[:16]) and torch.equal(out[32:], k[32:])
     pool.destroy()
+
+
+def test_owners_pins_and_lru_follow_the_oracle():
+    # Random walk over every allocator call; the library and the oracle must agree on each result, each error
+    # and the state of every page after each call.
+    n_pages = 24
+    pool = kvattn.kv_pool_create(n_pages, 16, 2, 64)
+    ref = orc.FreeList(n_pages)
+    rng = np.random.default_rng(23)
+    errs = {kvattn.KV_ERR_NOT_ALLOCATED: KeyError, kvattn.KV_ERR_PINNED: orc.PinnedError, kvattn.KV_ERR_INVALID: ValueError}
+    calls = [("free", kvattn.kv_free, ref.free), ("evict", kvattn.kv_evict, ref.evict), ("ref", kvattn.kv_ref, ref.ref),
+             ("pin", kvattn.kv_pin, ref.pin), ("unpin", kvattn.kv_unpin, ref.unpin), ("touch", kvattn.kv_touch, ref.touch)]
+    seen_errors = set()
+    for step in range(1500):
+        op = int(rng.integers(0, 9))
+        if op == 0:
+            n = int(rng.integers(0, 6))
+            want = ref.alloc(n)
+            if want is None:
+                with pytest.raises(kvattn.KvError) as e:
+                    kvattn.kv_alloc(pool, n)
+                assert e.value.status == kvattn.KV_ERR_OOM
+            else:
+                assert kvattn.kv_alloc(pool, n) == want
+        elif op == 7:
+            n = int(rng.integers(0, 4))
+            assert kvattn.kv_evict_lru(pool, n) == ref.evict_lru(n)
+        elif op == 8:
+            if rng.random() < 0.1:
+                assert kvattn.kv_unpin_all(pool) == ref.unpin_all()
+        else:
+            name, lib_fn, ref_fn = calls[op - 1]
+            # mostly live pages, sometimes a stray or repeated id
+            live = [p for p in range(n_pages) if ref.allocated[p]]
+            k = int(rng.integers(1, 4))
+            ids = [int(rng.choice(live)) if live and rng.random() < 0.9 else int(rng.integers(0, n_pages)) for _ in range(k)]
+            try:
+                ref_fn(list(ids))
+                expect = None
+            except (KeyError, orc.PinnedError, ValueError) as ex:
+                expect = type(ex)
+            if expect is None:
+                lib_fn(pool, ids)
+            else:
+                with pytest.raises(kvattn.KvError) as e:
+                    lib_fn(pool, ids)
+                assert errs[e.value.status] is expect, (name, ids, e.value.status)
+                seen_errors.add(e.value.status)
+        free, used, ev = kvattn.kv_pool_stats(pool)
+        assert (free, ev) == (ref.free_pages, ref.evicted_total)
+        for p in range(n_pages):
+            assert kvattn.kv_page_info(pool, p) == (int(ref.allocated[p]), ref.refs[p], ref.pins[p] if ref.allocated[p] else 0) \
+                or not ref.allocated[p]
+    assert seen_errors == set(errs)                                   # every kind of refusal was exercised
+    pool.destroy()

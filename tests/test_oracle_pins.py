@@ -328,3 +328,74 @@ def test_widen_is_exact():
     bits = np.array([0x0000, 0x3F80, 0xBF80, 0x4049, 0x0001, 0x7F7F], np.uint16)
     ref = synth.bits_to_bf16(bits).to(torch.float64).numpy()
     assert np.array_equal(orc.widen(bits), ref)
+
+
+# ------------------------------------------------ owners, pins, eviction order
+def test_shared_pages_return_with_their_last_owner():
+    fl = orc.FreeList(8)
+    parent = fl.alloc(3)                                          # [0, 1, 2]
+    for _ in range(2):                                            # two children read the parent's prefix
+        fl.ref(parent)
+    fl.free(parent)                                               # the parent is done: pages stay
+    assert fl.free_pages == 5 and all(fl.allocated[p] for p in parent)
+    fl.free(parent[:2])                                           # first child done with two of them
+    assert fl.free_pages == 5
+    fl.free(parent)                                               # second child: pages 0 and 1 go back, 2 has one owner left
+    assert fl.free_pages == 7 and not fl.allocated[0] and not fl.allocated[1] and fl.allocated[2]
+    assert fl.alloc(2) == [1, 0]                                  # last in, first out
+    with pytest.raises(KeyError):
+        fl.ref([5])                                               # not allocated
+
+
+def test_pinned_pages_are_never_evicted_and_unpin_all_is_the_fallback():
+    fl = orc.FreeList(6)
+    ids = fl.alloc(4)
+    fl.pin([ids[1]]); fl.pin([ids[1]]); fl.pin([ids[3]])          # pins are counted
+    with pytest.raises(orc.PinnedError):
+        fl.evict([ids[0], ids[1]])
+    assert fl.allocated[ids[0]]                                   # no partial effect
+    with pytest.raises(orc.PinnedError):
+        fl.free([ids[3]])                                         # the last owner cannot drop a pinned page
+    fl.unpin([ids[1]])
+    with pytest.raises(orc.PinnedError):
+        fl.evict([ids[1]])                                        # still pinned once
+    with pytest.raises(ValueError):
+        fl.unpin([ids[0]])                                        # was never pinned
+    assert fl.evict_lru(10) == [ids[0], ids[2]]                   # skips the pinned ones
+    assert fl.unpin_all() == 2
+    assert fl.evict_lru(10) == [ids[1], ids[3]] and fl.evicted_total == 4 and fl.free_pages == 6
+
+
+def test_lru_order_follows_alloc_and_touch():
+    fl = orc.FreeList(8)
+    a = fl.alloc(5)                                               # clock 1..5
+    fl.touch([a[0], a[2]])                                        # now the most recent
+    assert fl.evict_lru(2) == [a[1], a[3]]
+    b = fl.alloc(1)                                               # reuses a[3] (LIFO), newest of all
+    assert b == [a[3]]
+    assert fl.evict_lru(3) == [a[4], a[0], a[2]]
+    assert fl.evict_lru(3) == [a[3]] and fl.evict_lru(1) == []
+
+
+def test_free_list_invariants_under_random_operations():
+    rng = np.random.default_rng(17)
+    fl = orc.FreeList(16)
+    for _ in range(3000):
+        op = rng.integers(0, 8)
+        live = [p for p in range(16) if fl.allocated[p]]
+        pick = [int(p) for p in rng.choice(live, size=min(len(live), int(rng.integers(1, 4))), replace=False)] if live else []
+        try:
+            if op == 0: fl.alloc(int(rng.integers(0, 5)))
+            elif op == 1 and pick: fl.free(pick)
+            elif op == 2 and pick: fl.evict(pick)
+            elif op == 3 and pick: fl.ref(pick)
+            elif op == 4 and pick: fl.pin(pick)
+            elif op == 5 and pick: fl.unpin(pick)
+            elif op == 6 and pick: fl.touch(pick)
+            elif op == 7: fl.evict_lru(int(rng.integers(0, 3)))
+        except (orc.PinnedError, ValueError):
+            pass
+        alloc = {p for p in range(16) if fl.allocated[p]}
+        assert alloc.isdisjoint(fl.stack) and len(alloc) + len(fl.stack) == 16 and len(set(fl.stack)) == len(fl.stack)
+        assert all((fl.refs[p] >= 1) == (p in alloc) for p in range(16))
+        assert all(fl.pins[p] == 0 for p in fl.stack)             # nothing pinned is ever on the free list
