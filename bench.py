@@ -307,8 +307,12 @@ def extra_measurements(args, dev, peaks, flush):
     out = {}
     sections = set(x for x in args.sections.split(",") if x and x != "none")
     steps, warm = max(5, args.steps), 3
+    if "reuse" in sections:
+        out.update(reuse_vs_recompute(args, dev, peaks, flush))
     if not sections & {"decode", "append"}:
-        return mixed_measurement(args, dev, flush, steps, warm) if "mixed" in sections else out
+        if "mixed" in sections:
+            out.update(mixed_measurement(args, dev, flush, steps, warm))
+        return out
     # decode
     w = synth.WORKLOADS["decode_8b"]
     wl = DeviceWorkload(w, dev)
@@ -351,6 +355,51 @@ def extra_measurements(args, dev, peaks, flush):
     if "mixed" in sections:
         out.update(mixed_measurement(args, dev, flush, steps, warm))
     return out
+
+
+def reuse_vs_recompute(args, dev, peaks, flush):
+    """Long-document reuse (70B shape): extend over the reused prefix pages against the from-scratch prefill of
+    prefix+suffix that a cache miss costs (the kernel-level face of the paper's pipelined-vs-blocking gap)."""
+    from paper_2607_23815_b200 import kvattn
+    from paper_2607_23815_b200.workload import DeviceWorkload
+    w = synth.WORKLOADS["long_doc_70b"]
+    g = w.geom
+    wl = DeviceWorkload(w, dev)
+    e = wl.ext
+    ms_reuse, _ = time_steps(lambda _: wl.extend(), 5, 3, flush, 1)
+    t_reuse = statistics.mean(ms_reuse)
+    # the same sequences from scratch: prefix 0, every token is a query (K/V are already in the pages)
+    L = [p + x for p, x in zip(e.prefix, e.extend)]
+    q_full = torch.cat([synth.normal_bf16(wl.seed, synth.TAG_Q, e.uids[i], 0, L[i], g.n_q_heads, g.head_dim, dev)
+                        for i in range(len(L))])
+    out_full = torch.empty_like(q_full)
+    lse_full = torch.empty((q_full.shape[0], g.n_q_heads), dtype=torch.float32, device=dev)
+    i32 = lambda x: torch.tensor(x, dtype=torch.int32, device=dev)
+    cu, zero, lens = i32(np.concatenate([[0], np.cumsum(L)]).tolist()), i32([0] * len(L)), i32(L)
+    ws = torch.empty(kvattn.attn_workspace_bytes(wl.pool, g.n_q_heads, len(L), int(q_full.shape[0]), max(L), 0, 0),
+                     dtype=torch.uint8, device=dev)
+    fn = lambda _: kvattn.attn_extend(wl.pool, q_full, cu, e.block_tables, zero, lens, max(L), max(L), g.scale,
+                                      out_full, lse_full, ws)
+    ms_full, _ = time_steps(fn, 3, 1, flush, 1)
+    t_full = statistics.mean(ms_full)
+    # the last E rows of the recompute are the reuse run's rows: the invariant the paper relies on
+    r0, f0 = int(e.cu_q[1].item()), int(cu[1].item())
+    d_o = (out_full[f0 - e.extend[0]:f0].float() - e.out[:r0].float()).abs().max().item()
+    flops_reuse = e.flops(g)
+    flops_full = 4.0 * g.head_dim * g.n_q_heads * sum(l * (l + 1) // 2 for l in L)
+    res = {"reuse_vs_recompute": {
+        "workload": f"{w.name}: {w.n_extend} tuples, Hq={g.n_q_heads} Hkv={g.n_kv_heads}, prefix U{list(w.prefix_range)}, "
+                    f"extend U{list(w.extend_range)}",
+        "reuse_ms": round(t_reuse, 4), "reuse_tflops": round(flops_reuse / t_reuse / 1e9, 1),
+        "reuse_frac_of_measured_peak": round(flops_reuse / t_reuse / 1e9 / peaks["bf16_tflops"], 4),
+        "recompute_ms": round(t_full, 3), "recompute_tflops": round(flops_full / t_full / 1e9, 1),
+        "recompute_frac_of_measured_peak": round(flops_full / t_full / 1e9 / peaks["bf16_tflops"], 4),
+        "time_ratio": round(t_full / t_reuse, 2), "flop_ratio": round(flops_full / flops_reuse, 2),
+        "max_abs_diff_last_rows_tuple0": d_o}}
+    del q_full, out_full, lse_full, ws
+    wl.close(); del wl
+    torch.cuda.empty_cache()
+    return res
 
 
 def mixed_measurement(args, dev, flush, steps, warm):
@@ -426,8 +475,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=HEADLINE, choices=[k for k, v in synth.WORKLOADS.items() if v.n_extend])
     ap.add_argument("--cpu-sample", type=int, default=64, help="tuples in the CPU-oracle sample")
-    ap.add_argument("--sections", default="decode,append,mixed",
-                    help="extra measurements after the headline: comma list of decode, append, mixed (or 'none')")
+    ap.add_argument("--sections", default="decode,append,mixed,reuse",
+                    help="extra measurements after the headline: comma list of decode, append, mixed, reuse (or 'none')")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle legs (for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
