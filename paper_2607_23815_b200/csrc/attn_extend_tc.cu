@@ -11,12 +11,17 @@
 //               shared-memory stages; completion is signalled on mbarriers.
 //   warp 1      MMA issuer (one elected lane): S = Q K^T and O += P V on tcgen05 with accumulators in
 //               tensor memory; P is read straight from tensor memory (it overwrites S in place).
-//   warps 2, 3  idle (they give their registers to the softmax warps).
+//   warp 2      Q loader: one tensor-map (TMA) copy per 64-dim half brings a query tile into shared
+//               memory in the swizzled operand layout, as soon as the MMAs that read the previous
+//               item's tile have finished.
+//   warp 3      idle (warps 0-3 give most of their registers to the softmax warps).
 //   warps 4-7   softmax of query tile 0: one thread per row (= TMEM lane): masks, running max and
 //   warps 8-11  sum, exp2, P as bf16 back to TMEM, lazy rescale of O, final normalise + store.
 // The two query tiles ping-pong: while one tile's softmax runs, the tensor core works on the other.
 // All waits are bounded; on expiry the CTA records KV_ERR_TIMEOUT, drains its copies, frees its
 // tensor memory and returns.
+#include <cuda.h>  // CUtensorMap and its enums (types only: the encoder is looked up at run time)
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -173,7 +178,7 @@ struct __align__(1024) TcSmem {
   unsigned char q[2][TcCfg<D>::kTileBytes];
   unsigned char kv[TcCfg<D>::kStages][TcCfg<D>::kTileBytes];
   unsigned long long kv_full[TcCfg<D>::kStages], kv_empty[TcCfg<D>::kStages];
-  unsigned long long q_full[2], s_full[2], p_full[2], o_full[2];
+  unsigned long long q_full[2], q_empty[2], s_full[2], p_full[2], o_full[2];
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -232,7 +237,7 @@ __device__ __forceinline__ int item_index(int round) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcArgs a) {
+__global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap q_map) {
   using Cfg = TcCfg<D>;
   extern __shared__ unsigned char smem_raw[];
   TcSmem<D>& sm = *reinterpret_cast<TcSmem<D>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -246,7 +251,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       mbar_init(smem_u32(&sm.kv_empty[s]), 1);
     }
     for (int t = 0; t < 2; ++t) {
-      mbar_init(smem_u32(&sm.q_full[t]), 128);  // every softmax thread stored its part of the Q tile
+      mbar_init(smem_u32(&sm.q_full[t]), 1);    // the Q tile's bytes have landed (transaction count)
+      mbar_init(smem_u32(&sm.q_empty[t]), 1);   // tensor core finished the item's last S: the Q buffer may be refilled
       mbar_init(smem_u32(&sm.s_full[t]), 1);    // tensor core finished S (and everything issued before it)
       mbar_init(smem_u32(&sm.p_full[t]), 128);  // every softmax thread wrote its row of P
       mbar_init(smem_u32(&sm.o_full[t]), 1);    // tensor core finished the item's last PV
@@ -266,7 +272,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
 
   if (warp == 0) {
     // =============================== producer =============================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     const char* kpool = reinterpret_cast<const char*>(a.pool.k);
     const char* vpool = reinterpret_cast<const char*>(a.pool.v);
     uint32_t loads = 0;  // stage loads issued so far (ring position)
@@ -321,12 +327,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
     // One thread issues every MMA of the CTA.  Per KV tile j and query tile t:  O_t (+)= P_t V(j) as soon as
     // the softmax warps have written P_t, then S_t = Q_t K(j+1)^T into the columns P_t occupied (the tensor
     // core runs MMAs in issue order), so the other tile's MMAs fill the time this tile's softmax takes.
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     const uint32_t q_lo0 = (smem_u32(sm.q[0]) >> 4) | (1u << 16);             // low descriptor words: LBO field 16 B
     const uint32_t k_lo0 = (smem_u32(sm.kv[0]) >> 4) | (1u << 16);
     const uint32_t v_lo0 = (smem_u32(sm.kv[0]) >> 4) | ((1024u >> 4) << 16);  // V tiles: LBO = 64-dim half
     const uint32_t bar_s_full = smem_u32(&sm.s_full[0]), bar_p_full = smem_u32(&sm.p_full[0]);
     const uint32_t bar_q_full = smem_u32(&sm.q_full[0]), bar_o_full = smem_u32(&sm.o_full[0]);
+    const uint32_t bar_q_empty = smem_u32(&sm.q_empty[0]);
     uint32_t loads = 0;                 // ring position, mirrors the producer
     uint32_t steps[2] = {0, 0};         // softmax steps per tile so far (phase of p_full)
     uint32_t items_done[2] = {0, 0};    // items per tile so far (phase of q_full)
@@ -352,6 +359,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
           if (elect_one_sync()) {
             issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + stage * (Cfg::kTileBytes >> 4));
             mma_commit(bar_s_full + 8 * t);
+            if (it.n_kv[t] == 1) mma_commit(bar_q_empty + 8 * t);
           }
           __syncwarp();
         }
@@ -383,6 +391,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
               if (j + 1 < it.n_kv[t]) {
                 issue_s_mmas<D>(tmem + t * 128, q_lo0 + t * (Cfg::kTileBytes >> 4), k_lo0 + k_stage * (Cfg::kTileBytes >> 4));
                 mma_commit(bar_s_full + 8 * t);
+                if (j + 2 == it.n_kv[t]) mma_commit(bar_q_empty + 8 * t);  // that was the item's last S of this tile
               } else {
                 mma_commit(bar_o_full + 8 * t);
               }
@@ -399,110 +408,96 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       ok = __all_sync(0xffffffffu, ok);
     }
+  } else if (warp == 2) {
+    // =============================== Q loader ============================================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    uint32_t fills[2] = {0, 0};  // tiles loaded so far per buffer (phase of q_empty)
+    bool ok = true;
+    Item it;
+    for (int round = 0; ok && fetch_item(a, item_index(round), n_total, it); ++round) {
+      if (it.ld_tiles == 0) continue;
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        if (it.n_kv[t] == 0 || !ok) continue;
+        if (lane == 0) {
+          // the buffer is free once the previous item's last S of this tile has been computed
+          ok = mbar_wait(smem_u32(&sm.q_empty[t]), (fills[t] & 1) ^ 1, abortp);
+          if (ok) {
+            const uint32_t full = smem_u32(&sm.q_full[t]);
+            mbar_arrive_expect_tx(full, Cfg::kTileBytes);
+            const int tok0 = it.row0 + ((it.tp * 256 + t * 128) >> a.lg_group);
+#pragma unroll
+            for (int h = 0; h < Cfg::kHalves; ++h)
+              tma_load_3d(smem_u32(sm.q[t]) + h * Cfg::kQHalfStride, &q_map, h * 64, it.kvh * a.group, tok0, full);
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        ++fills[t];
+      }
+    }
   } else if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");  // idle warps
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");  // idle warp
   } else {
     // =============================== softmax warpgroups ======================================
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     const int t = (warp - 4) >> 2;                 // query tile of this warpgroup (warps 4-7: tile 0, 8-11: tile 1)
     const int w4 = warp & 3;                       // TMEM lane quarter this warp may access
     const int m = w4 * 32 + lane;                  // row inside the tile
     const uint32_t lane_base = tmem + ((uint32_t)(w4 * 32) << 16);
     const uint32_t s_addr = lane_base + t * 128, o_addr = lane_base + 256 + t * 128;
     const uint32_t bar_s_full = smem_u32(&sm.s_full[t]), bar_o_full = smem_u32(&sm.o_full[t]);
-    const uint32_t bar_q_full = smem_u32(&sm.q_full[t]), bar_p_full = smem_u32(&sm.p_full[t]);
+    const uint32_t bar_p_full = smem_u32(&sm.p_full[t]);
     const int G = a.group, lg = a.lg_group, Hq = a.n_q_heads;
     uint32_t steps = 0, items_done = 0;            // phases of s_full / p_full and of q_full / o_full
     bool ok = true;
 
-    // Q rows of this warp, 16-byte chunks: iteration i covers rows w4*32 + i*RPI .. and chunk lane % CPR
-    constexpr int CPR = D / 8, RPI = 32 / CPR, QIT = 32 / RPI;  // chunks per row, rows per iteration, iterations
-    auto q_load = [&](const Item& qi, uint4 (&qv)[QIT]) {        // global -> registers (coalesced 16-byte loads)
-#pragma unroll
-      for (int i = 0; i < QIT; ++i) {
-        const int row = w4 * 32 + i * RPI + lane / CPR, chunk = lane % CPR;
-        const int rg = qi.tp * 256 + t * 128 + row;
+    // The item records are read where they are needed (they stay in L1) instead of being carried in registers
+    // through the softmax loop, which needs the registers for the score row.
+    for (int round = 0; ok; ++round) {
+      int n_t, limit;
+      bool valid;
+      int64_t orow_idx;
+      {
+        Item it;
+        if (!fetch_item(a, item_index(round), n_total, it)) break;
+        if (it.ld_tiles == 0) continue;
+        n_t = it.n_kv[t];
+        if (n_t == 0) continue;
+        const int rg = it.tp * 256 + t * 128 + m;
         const int tok = rg >> lg;
-        qv[i] = make_uint4(0, 0, 0, 0);
-        if (tok < qi.E)
-          qv[i] = __ldg(reinterpret_cast<const uint4*>(a.q + ((int64_t)(qi.row0 + tok) * Hq + qi.kvh * G + (rg & (G - 1))) * D) + chunk);
+        valid = tok < it.E;
+        limit = valid ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
+        orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));
       }
-    };
-    auto q_store = [&](const uint4 (&qv)[QIT]) {  // registers -> shared, swizzled K-major operand layout
-#pragma unroll
-      for (int i = 0; i < QIT; ++i) {
-        const int row = w4 * 32 + i * RPI + lane / CPR, chunk = lane % CPR;
-        *reinterpret_cast<uint4*>(sm.q[t] + (chunk >> 3) * Cfg::kQHalfStride + (row >> 3) * 1024 + (row & 7) * 128 +
-                                  (((chunk & 7) ^ (row & 7)) << 4)) = qv[i];
-      }
-      fence_proxy_async_smem();  // make the generic-proxy stores visible to the tensor core's reads
-      mbar_arrive(bar_q_full);
-    };
-    bool q_stored = false;  // this item's Q tile is already in shared memory (stored during the previous item)
-    Item nxt;
-    bool has_nxt = fetch_item(a, item_index(0), n_total, nxt);
-    for (int round = 0; ok && has_nxt; ++round) {
-      const Item it = nxt;
-      has_nxt = fetch_item(a, item_index(round + 1), n_total, nxt);
-      if (it.ld_tiles == 0) continue;
-      const int n_t = it.n_kv[t];
-      if (n_t == 0) continue;
-      if (!q_stored) {
-        uint4 qv[QIT];
-        q_load(it, qv);
-        q_store(qv);
-      }
-      q_stored = false;
-      const bool preload = has_nxt && nxt.n_kv[t] > 0;
-      const int rg = it.tp * 256 + t * 128 + m;
-      const int tok = rg >> lg;
-      const bool valid = tok < it.E;
-      const int limit = valid ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
       float m_run = -INFINITY, l_run = 0.f;
 
       for (int j = 0; j < n_t; ++j) {
-        // The next item's Q rows are fetched while this thread waits for the item's last S; once that S is
-        // there, every MMA that reads this tile's Q buffer has finished and the buffer can be refilled, so the
-        // next item's first S overlaps this item's last softmax step and epilogue.
-        const bool refill = preload && j + 1 == n_t;
-        uint4 qn[QIT];
-        if (refill) q_load(nxt, qn);
         ok = mbar_wait(bar_s_full, steps & 1, abortp);
         ++steps;
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
-        if (refill) {
-          q_store(qn);
-          q_stored = true;
-        }
-        // Two passes over the 128 score columns, 64 at a time, to keep the live registers low:
-        // pass 1 finds the row maximum, pass 2 re-reads the scores, exponentiates and writes P.
+        // One trip to tensor memory: the row's 128 scores are read into registers, reduced to the row
+        // maximum, exponentiated in place and written back as bf16 P.
         const int kv0 = j * 128;
         const bool ragged = kv0 + 128 > limit;  // diagonal / last tile: keys past the row's limit are hidden
-        auto load_half = [&](int h, uint32_t (&sr)[2][32]) {
-          tmem_ld32(s_addr + h * 64, sr[0]);
-          tmem_ld32(s_addr + h * 64 + 32, sr[1]);
-          tmem_wait_ld();
-          if (ragged) {
+        uint32_t sr[4][32];
 #pragma unroll
-            for (int c = 0; c < 2; ++c)
+        for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr[c]);
+        tmem_wait_ld();
+        if (ragged) {
 #pragma unroll
-              for (int i = 0; i < 32; ++i)
-                if (kv0 + h * 64 + c * 32 + i >= limit) sr[c][i] = 0xff800000u;  // -inf by select: NaN-safe
-          }
-        };
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+              if (kv0 + c * 32 + i >= limit) sr[c][i] = 0xff800000u;  // -inf by select: NaN-safe
+        }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t sr[2][32];
-          load_half(h, sr);
+        for (int c = 0; c < 4; ++c)
 #pragma unroll
-          for (int c = 0; c < 2; ++c)
-#pragma unroll
-            for (int i = 0; i < 32; i += 2)
-              mx4[2 * c + ((i >> 1) & 1)] = fmax3(mx4[2 * c + ((i >> 1) & 1)], __uint_as_float(sr[c][i]), __uint_as_float(sr[c][i + 1]));
-        }
+          for (int i = 0; i < 32; i += 2)
+            mx4[c] = fmax3(mx4[c], __uint_as_float(sr[c][i]), __uint_as_float(sr[c][i + 1]));
         const float mx = fmax3(fmaxf(mx4[0], mx4[1]), mx4[2], mx4[3]) * a.scale_log2;
         const float m_new = fmaxf(m_run, mx);
         const bool grow = m_new > m_run + kRescaleThreshold;  // also true on the first tile (m_run = -inf)
@@ -512,14 +507,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
           // has finished: the S this step waited for was committed after it)
           const float alpha = grow ? exp2f(m_run - m_new) : 1.f;
           l_run *= alpha;
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c) {
-            uint32_t orow[32];
-            tmem_ld32(o_addr + c * 32, orow);
+#pragma unroll 1
+          for (int c = 0; c < D / 16; ++c) {
+            uint32_t orow[16];
+            tmem_ld16(o_addr + c * 16, orow);
             tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) orow[i] = __float_as_uint(__uint_as_float(orow[i]) * alpha);
-            tmem_st32(o_addr + c * 32, orow);
+            for (int i = 0; i < 16; ++i) orow[i] = __float_as_uint(__uint_as_float(orow[i]) * alpha);
+            tmem_st16(o_addr + c * 16, orow);
           }
         }
         m_run = m_use;
@@ -527,25 +522,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         const float2 sc2 = make_float2(a.scale_log2, a.scale_log2), nm2 = make_float2(neg_m, neg_m);
         float2 ls2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          uint32_t sr[2][32];
-          load_half(h, sr);
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[c][2 * i]), __uint_as_float(sr[c][2 * i + 1])), sc2, nm2);
-              float2 pr;
-              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pr.x) : "f"(x.x));
-              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pr.y) : "f"(x.y));
-              ls2[i & 1] = __fadd2_rn(ls2[i & 1], pr);
-              asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[i]) : "f"(pr.y), "f"(pr.x));
-            }
-            // P (bf16 pairs) overwrites score columns that have already been read: columns [32h+16c, +16)
-            // lie below the 64-column half being processed, or inside the part of it held in registers
-            tmem_st16(s_addr + h * 32 + c * 16, pk);
+          for (int i = 0; i < 16; ++i) {
+            const float2 x = __ffma2_rn(make_float2(__uint_as_float(sr[c][2 * i]), __uint_as_float(sr[c][2 * i + 1])), sc2, nm2);
+            float2 pr;
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pr.x) : "f"(x.x));
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(pr.y) : "f"(x.y));
+            ls2[i & 1] = __fadd2_rn(ls2[i & 1], pr);
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[i]) : "f"(pr.y), "f"(pr.x));
           }
+          // P (bf16 pairs) goes over score columns [16c, 16c+16): all scores are in registers by now
+          tmem_st16(s_addr + c * 16, pk);
         }
         l_run += (ls2[0].x + ls2[0].y) + (ls2[1].x + ls2[1].y);
         tmem_wait_st();
@@ -561,7 +550,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       if (!ok) break;
       tc_fence_after_sync();
       const float inv = 1.f / l_run;
-      const int64_t orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));
 #pragma unroll
       for (int c = 0; c < D / 32; ++c) {
         uint32_t orow[32];
@@ -613,8 +601,33 @@ bool extend_tc_supported(const kv_pool_t* p, int n_q_heads) {
   return g == 1 || g == 2 || g == 4 || g == 8;
 }
 
+// Tensor map over Q [total_q][Hq][D] (bf16): a box is one 64-dim half of a query tile, that is 128/G tokens x the
+// G heads of one KV head x 64 dims, written to shared memory with the 128-byte swizzle the MMA expects.  Rows past
+// the end of Q read as zeros.
+static kv_status_t make_q_map(CUtensorMap* map, const void* q, int total_q, int n_q_heads, int head_dim, int group) {
+  typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  static encode_fn encode = nullptr;
+  if (encode == nullptr) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    KV_CUDA_OK(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres));
+    if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return KV_ERR_CUDA;
+    encode = reinterpret_cast<encode_fn>(fn);
+  }
+  const cuuint64_t dims[3] = {(cuuint64_t)head_dim, (cuuint64_t)n_q_heads, (cuuint64_t)total_q};
+  const cuuint64_t strides[2] = {(cuuint64_t)head_dim * 2, (cuuint64_t)n_q_heads * head_dim * 2};
+  const cuuint32_t box[3] = {64, (cuuint32_t)group, (cuuint32_t)(128 / group)};
+  const cuuint32_t elem_strides[3] = {1, 1, 1};
+  const CUresult r = encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(q), dims, strides, box, elem_strides,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? KV_OK : KV_ERR_INVALID;
+}
+
 template <int D>
-static kv_status_t launch_tc(const TcArgs& a, int n_items_bound, int cta_cap, cudaStream_t st) {
+static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int n_items_bound, int cta_cap, cudaStream_t st) {
   static int sm_count = 0;
   if (sm_count == 0) {
     int dev = 0;
@@ -629,7 +642,7 @@ static kv_status_t launch_tc(const TcArgs& a, int n_items_bound, int cta_cap, cu
   }
   int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
   if (cta_cap > 0 && grid > cta_cap) grid = cta_cap;  // leave the other SMs to work that runs beside this kernel
-  attn_extend_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(a);
+  attn_extend_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(a, q_map);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
   return KV_OK;
@@ -642,6 +655,12 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   const size_t need = extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch, total_q, max_total_len);
   if (workspace == nullptr || workspace_bytes < need) return KV_ERR_WORKSPACE;
   const int G = n_q_heads / p->n_kv_heads;
+  if ((reinterpret_cast<uintptr_t>(q) & 15) != 0) return KV_ERR_INVALID;
+  CUtensorMap q_map;
+  {
+    const kv_status_t ms = make_q_map(&q_map, q, total_q, n_q_heads, p->head_dim, G);
+    if (ms != KV_OK) return ms;
+  }
   int lg = 0;
   while ((1 << lg) < G) ++lg;
   int* n_items = reinterpret_cast<int*>(workspace);
@@ -673,8 +692,8 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   a.n_items = n_items;
   const int64_t bound = (int64_t)batch * max_tp * p->n_kv_heads;
   const int n_bound = bound > (1 << 30) ? (1 << 30) : (int)bound;
-  if (p->head_dim == 128) return launch_tc<128>(a, n_bound, cta_cap, st);
-  return launch_tc<64>(a, n_bound, cta_cap, st);
+  if (p->head_dim == 128) return launch_tc<128>(a, q_map, n_bound, cta_cap, st);
+  return launch_tc<64>(a, q_map, n_bound, cta_cap, st);
 }
 
 }  // namespace kvattn
