@@ -5,18 +5,20 @@
 // share a KV head share every K/V tile that is brought on chip (GQA) and the causal diagonal is
 // only 128/G tokens wide.  One persistent CTA per SM walks a cost-sorted item list.
 //
-// Roles (warp-specialised, 12 warps):
-//   warp 0      producer: per 128-token KV tile, one 1-D bulk copy per 16-token page block
+// Roles (warp-specialised, 16 warps):
+//   warps 0-3   softmax of query tile 0: one thread per row (= TMEM lane): masks, running max and
+//   warps 4-7   softmax of query tile 1: sum, exp2, P as bf16 back to TMEM, lazy rescale of O.
+//   warps 8-11  epilogue of both tiles: O / l -> bf16 -> global, while the softmax warps are already
+//               at the next item.
+//   warp 12     producer: per 128-token KV tile, one 1-D bulk copy per 16-token page block
 //               (the pool keeps blocks in the MMA's 128-byte-swizzle operand layout) into a ring of
 //               shared-memory stages; completion is signalled on mbarriers.
-//   warp 1      MMA issuer (one elected lane): S = Q K^T and O += P V on tcgen05 with accumulators in
+//   warp 13     MMA issuer (one elected lane): S = Q K^T and O += P V on tcgen05 with accumulators in
 //               tensor memory; P is read straight from tensor memory (it overwrites S in place).
-//   warp 2      Q loader: one tensor-map (TMA) copy per 64-dim half brings a query tile into shared
+//   warp 14     Q loader: one tensor-map (TMA) copy per 64-dim half brings a query tile into shared
 //               memory in the swizzled operand layout, as soon as the MMAs that read the previous
 //               item's tile have finished.
-//   warp 3      idle (warps 0-3 give most of their registers to the softmax warps).
-//   warps 4-7   softmax of query tile 0: one thread per row (= TMEM lane): masks, running max and
-//   warps 8-11  sum, exp2, P as bf16 back to TMEM, lazy rescale of O, final normalise + store.
+//   warp 15     idle (launched for the registers it hands to the others).
 // The two query tiles ping-pong: while one tile's softmax runs, the tensor core works on the other.
 // All waits are bounded; on expiry the CTA records KV_ERR_TIMEOUT, drains its copies, frees its
 // tensor memory and returns.
@@ -28,7 +30,11 @@
 namespace kvattn {
 using namespace ptx;
 
-constexpr int kTcThreads = 384;  // warp 0: producer, warps 1-3: idle, warps 4-11: two softmax warpgroups
+// The roles' register budgets are set with setmaxnreg.  What the warps hold afterwards must not exceed what the
+// CTA was launched with (512 threads x 128 registers), in total and per scheduler (warp index mod 4):
+// 8 x 192 (softmax) + 4 x 72 (epilogue) + 56 + 56 + 40 + 24 = 2000 <= 2048 per lane.
+constexpr int kTcThreads = 512;
+constexpr int kWarpEpilogue = 8, kWarpProducer = 12, kWarpMma = 13, kWarpQ = 14;
 constexpr int kPlanBuckets = 2048;
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more than this
 
@@ -46,6 +52,7 @@ struct TcArgs {
   float* lse;
   const int4* items;   // two int4 per entry (see ItemRec), cost-sorted
   const int* n_items;  // number of valid entries in items
+  int* next_item;      // work counter: the next item of the global list nobody has taken yet
 };
 
 // ------------------------------------------------------------------------------------------
@@ -92,7 +99,9 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
                                                               const int* __restrict__ cu_q, int batch, int max_tp,
                                                               int lg, int max_steps, int capacity, int max_pages,
                                                               int* status, int4* __restrict__ items,
-                                                              int* __restrict__ n_items) {
+                                                              int* __restrict__ n_items, int* __restrict__ next_item,
+                                                              int first_free_item) {
+  if (threadIdx.x == 0) *next_item = first_free_item;  // the CTAs start on items 0 .. grid-1 without asking
   __shared__ int hist[kPlanBuckets];
   for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
   __syncthreads();
@@ -178,7 +187,12 @@ struct __align__(1024) TcSmem {
   unsigned char q[2][TcCfg<D>::kTileBytes];
   unsigned char kv[TcCfg<D>::kStages][TcCfg<D>::kTileBytes];
   unsigned long long kv_full[TcCfg<D>::kStages], kv_empty[TcCfg<D>::kStages];
-  unsigned long long q_full[2], q_empty[2], s_full[2], p_full[2], o_full[2];
+  unsigned long long q_full[2], q_empty[2], s_full[2], p_full[2], o_full[2], o_empty[2], l_full[2];
+  // Item queue of the CTA: the producer takes items off the global list (heaviest first, whoever is free
+  // takes the next) and announces them here; every role walks the same sequence.
+  unsigned long long sched_full[4], sched_empty[4];
+  int sched_idx[4];
+  float inv_l[2][2][128];  // [tile][item parity][row]: 1 / row sum, handed from the softmax to the epilogue warps
   uint32_t tmem_base;
   int abort_flag;
 };
@@ -231,16 +245,17 @@ __device__ __forceinline__ void issue_pv_mmas(uint32_t o_tmem, uint32_t p_tmem, 
     if (p < np) mma_ts(o_tmem, p_tmem + p * 8, make_desc(kHiV, v_lo + p * (D * 2)), idesc, 1u);
 }
 
-// item sequence of one CTA: boustrophedon over the sorted list, so that heavy and light items alternate
-__device__ __forceinline__ int item_index(int round) {
-  return (round & 1) ? round * gridDim.x + (gridDim.x - 1 - blockIdx.x) : round * gridDim.x + blockIdx.x;
-}
-
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap q_map) {
   using Cfg = TcCfg<D>;
   extern __shared__ unsigned char smem_raw[];
-  TcSmem<D>& sm = *reinterpret_cast<TcSmem<D>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  // Dynamic shared memory starts on a 1024-byte boundary (this kernel has no static shared memory); the swizzled
+  // operand tiles need that.  Checked instead of padded for: the tiles leave no room for padding.
+  if ((smem_u32(smem_raw) & 1023u) != 0) {
+    if (threadIdx.x == 0) report(a.pool.status, KV_ERR_CUDA);
+    return;
+  }
+  TcSmem<D>& sm = *reinterpret_cast<TcSmem<D>*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abortp = &sm.abort_flag;
 
@@ -250,16 +265,22 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       mbar_init(smem_u32(&sm.kv_full[s]), 1);
       mbar_init(smem_u32(&sm.kv_empty[s]), 1);
     }
+    for (int s4 = 0; s4 < 4; ++s4) {
+      mbar_init(smem_u32(&sm.sched_full[s4]), 1);    // the producer wrote the slot
+      mbar_init(smem_u32(&sm.sched_empty[s4]), 14);  // MMA warp, Q loader, 8 softmax and 4 epilogue warps have read it
+    }
     for (int t = 0; t < 2; ++t) {
       mbar_init(smem_u32(&sm.q_full[t]), 1);    // the Q tile's bytes have landed (transaction count)
       mbar_init(smem_u32(&sm.q_empty[t]), 1);   // tensor core finished the item's last S: the Q buffer may be refilled
       mbar_init(smem_u32(&sm.s_full[t]), 1);    // tensor core finished S (and everything issued before it)
       mbar_init(smem_u32(&sm.p_full[t]), 128);  // every softmax thread wrote its row of P
       mbar_init(smem_u32(&sm.o_full[t]), 1);    // tensor core finished the item's last PV
+      mbar_init(smem_u32(&sm.o_empty[t]), 128); // every epilogue thread has read its row of O: the next item may overwrite it
+      mbar_init(smem_u32(&sm.l_full[t]), 128);  // every softmax thread has published 1 / row sum
     }
     fence_mbar_init();
   }
-  if (warp == 0) {
+  if (warp == kWarpProducer) {
     tmem_alloc(smem_u32(&sm.tmem_base), 512);
     tmem_relinquish();
   }
@@ -269,19 +290,48 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
   const uint32_t tmem = sm.tmem_base;
   const int n_total = __ldg(a.n_items) * a.pool.n_kv_heads;
   const int Hkv = a.pool.n_kv_heads;
+  // Round r of this CTA works on item sched_get(r) of the global list (>= n_total: no more work).  A warp
+  // calls sched_release(r) once it no longer needs the slot.
+  auto sched_get = [&](int round) -> int {
+    const bool got = mbar_wait(smem_u32(&sm.sched_full[round & 3]), (round >> 2) & 1, abortp);
+    const int idx = *reinterpret_cast<volatile int*>(&sm.sched_idx[round & 3]);
+    return got ? idx : 0x7fffffff;
+  };
+  auto sched_release = [&](int round) {
+    __syncwarp();
+    if (lane == 0) mbar_arrive(smem_u32(&sm.sched_empty[round & 3]));
+  };
 
-  if (warp == 0) {
+  if (warp == kWarpProducer) {
     // =============================== producer =============================================
     asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
     const char* kpool = reinterpret_cast<const char*>(a.pool.k);
     const char* vpool = reinterpret_cast<const char*>(a.pool.v);
     uint32_t loads = 0;  // stage loads issued so far (ring position)
     bool ok = true;
-    Item nxt;
-    bool has_nxt = fetch_item(a, item_index(0), n_total, nxt);
-    for (int round = 0; ok && has_nxt; ++round) {
-      const Item it = nxt;
-      has_nxt = fetch_item(a, item_index(round + 1), n_total, nxt);  // next record is in flight during this item
+    // Announces item idx as round r (waits until every reader is done with the slot's previous round).
+    auto announce = [&](int r, int idx) {
+      if (lane == 0) {
+        ok = mbar_wait(smem_u32(&sm.sched_empty[r & 3]), ((r >> 2) & 1) ^ 1, abortp);
+        *reinterpret_cast<volatile int*>(&sm.sched_idx[r & 3]) = idx;
+        mbar_arrive(smem_u32(&sm.sched_full[r & 3]));
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+    };
+    int cur = blockIdx.x;
+    announce(0, cur);
+    for (int round = 0; ok && cur < n_total; ++round) {
+      // The next item is taken and announced one item ahead, so that nobody waits for the counter.  (Taking it
+      // two items ahead would hide the counter's latency from this warp too, but an item that is committed early
+      // cannot go to a CTA that runs out of work: measured slower.)
+      int nxt_idx = 0;
+      if (lane == 0) nxt_idx = atomicAdd(a.next_item, 1);
+      nxt_idx = __shfl_sync(0xffffffffu, nxt_idx, 0);
+      announce(round + 1, nxt_idx);
+      Item it;
+      fetch_item(a, cur, n_total, it);
+      cur = nxt_idx;
+      if (!ok) break;
       const int* bt = a.block_tables + (int64_t)it.seq * a.max_pages;
       const size_t head_off = (size_t)it.kvh * Cfg::kBlockBytes;
       for (int j = 0; j < it.ld_tiles && ok; ++j) {
@@ -322,7 +372,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         }
       }
     }
-  } else if (warp == 1) {
+  } else if (warp == kWarpMma) {
     // =============================== MMA issuer ===========================================
     // One thread issues every MMA of the CTA.  Per KV tile j and query tile t:  O_t (+)= P_t V(j) as soon as
     // the softmax warps have written P_t, then S_t = Q_t K(j+1)^T into the columns P_t occupied (the tensor
@@ -333,16 +383,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
     const uint32_t v_lo0 = (smem_u32(sm.kv[0]) >> 4) | ((1024u >> 4) << 16);  // V tiles: LBO = 64-dim half
     const uint32_t bar_s_full = smem_u32(&sm.s_full[0]), bar_p_full = smem_u32(&sm.p_full[0]);
     const uint32_t bar_q_full = smem_u32(&sm.q_full[0]), bar_o_full = smem_u32(&sm.o_full[0]);
-    const uint32_t bar_q_empty = smem_u32(&sm.q_empty[0]);
+    const uint32_t bar_q_empty = smem_u32(&sm.q_empty[0]), bar_o_empty = smem_u32(&sm.o_empty[0]);
+    uint32_t o_uses[2] = {0, 0};        // items per tile whose PV has started (phase of o_empty)
+    bool early0 = false;                // tile 0's first S of the coming item has been issued already
     uint32_t loads = 0;                 // ring position, mirrors the producer
     uint32_t steps[2] = {0, 0};         // softmax steps per tile so far (phase of p_full)
     uint32_t items_done[2] = {0, 0};    // items per tile so far (phase of q_full)
     bool ok = true;
     Item nxt;
-    bool has_nxt = fetch_item(a, item_index(0), n_total, nxt);
+    bool has_nxt = fetch_item(a, sched_get(0), n_total, nxt);
     for (int round = 0; ok && has_nxt; ++round) {
       const Item it = nxt;
-      has_nxt = fetch_item(a, item_index(round + 1), n_total, nxt);
+      has_nxt = fetch_item(a, sched_get(round + 1), n_total, nxt);
+      sched_release(round);
       if (it.ld_tiles == 0) continue;
       {
         // The whole warp runs this control flow (all values are warp-uniform); one elected lane issues.
@@ -353,6 +406,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
           if (!ok || it.n_kv[t] == 0) continue;
+          if (t == 0 && early0) {
+            early0 = false;
+            continue;
+          }
           ok = mbar_wait(bar_q_full + 8 * t, items_done[t] & 1, abortp);
           ++items_done[t];
           if (!ok) continue;
@@ -384,6 +441,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
             if (j >= it.n_kv[t]) continue;
             ok = mbar_wait(bar_p_full + 8 * t, steps[t] & 1, abortp);
             ++steps[t];
+            if (ok && j == 0) {  // the first PV overwrites O: the previous item's rows must have been read out
+              ok = mbar_wait(bar_o_empty + 8 * t, (o_uses[t] & 1) ^ 1, abortp);
+              ++o_uses[t];
+            }
             if (!ok) break;
             tc_fence_after_sync();
             if (elect_one_sync()) {
@@ -397,6 +458,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
               }
             }
             __syncwarp();
+            if (t == 0 && j + 1 == it.n_kv[0] && has_nxt && nxt.n_kv[0] > 0 && nxt.ld_tiles > 0) {
+              // Tile 0 is done with this item while tile 1 still has a step or more to go: if the next item's Q
+              // tile and first K tile are already there, its first S is issued now instead of after tile 1.
+              const uint32_t k0 = loads + (more ? 0 : 0) + 2 * (uint32_t)(it.ld_tiles - 1 - j) - (more ? 1 : 0);
+              const uint32_t st0 = k0 % Cfg::kStages;
+              if (__all_sync(0xffffffffu, mbar_test_wait(bar_q_full, items_done[0] & 1) &&
+                                              mbar_test_wait(smem_u32(&sm.kv_full[st0]), (k0 / Cfg::kStages) & 1))) {
+                ++items_done[0];
+                early0 = true;
+                if (elect_one_sync()) {
+                  issue_s_mmas<D>(tmem, q_lo0, k_lo0 + st0 * (Cfg::kTileBytes >> 4));
+                  mma_commit(bar_s_full);
+                  if (nxt.n_kv[0] == 1) mma_commit(bar_q_empty);
+                }
+                __syncwarp();
+              }
+            }
           }
           if (!ok) break;
           if (elect_one_sync()) {
@@ -408,13 +486,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       ok = __all_sync(0xffffffffu, ok);
     }
-  } else if (warp == 2) {
+  } else if (warp == kWarpQ) {
     // =============================== Q loader ============================================
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;");
     uint32_t fills[2] = {0, 0};  // tiles loaded so far per buffer (phase of q_empty)
     bool ok = true;
     Item it;
-    for (int round = 0; ok && fetch_item(a, item_index(round), n_total, it); ++round) {
+    for (int round = 0; ok && fetch_item(a, sched_get(round), n_total, it); ++round) {
+      sched_release(round);
       if (it.ld_tiles == 0) continue;
 #pragma unroll
       for (int t = 0; t < 2; ++t) {
@@ -434,21 +513,112 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         ok = __shfl_sync(0xffffffffu, ok, 0);
         ++fills[t];
       }
+      // the next item's query tiles are asked into L2 now, a whole item ahead of their copy to shared memory
+      Item nx;
+      if (fetch_item(a, sched_get(round + 1), n_total, nx) && nx.ld_tiles > 0 && lane == 0) {
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+          if (nx.n_kv[t] == 0) continue;
+          const int tok0 = nx.row0 + ((nx.tp * 256 + t * 128) >> a.lg_group);
+#pragma unroll
+          for (int h = 0; h < Cfg::kHalves; ++h) tma_prefetch_3d(&q_map, h * 64, nx.kvh * a.group, tok0);
+        }
+      }
     }
-  } else if (warp < 4) {
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");  // idle warp
+  } else if (warp == 15) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 24;");  // idle warp
+  } else if (warp >= kWarpEpilogue) {
+    // =============================== epilogue warpgroup ====================================
+    // One thread per row (= TMEM lane), both tiles in turn: O / l -> bf16 -> global.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+    const int w4 = warp & 3;
+    const int m = w4 * 32 + lane;
+    const uint32_t lane_base = tmem + ((uint32_t)(w4 * 32) << 16);
+    const int G = a.group, lg = a.lg_group, Hq = a.n_q_heads;
+    uint32_t done[2] = {0, 0};  // items finished per tile (phase of o_full / l_full, parity of inv_l)
+    bool ok = true;
+    Item it;
+    for (int round = 0; ok && fetch_item(a, sched_get(round), n_total, it); ++round) {
+      sched_release(round);
+      if (it.ld_tiles == 0) continue;
+#pragma unroll
+      for (int t = 0; t < 2; ++t) {
+        if (it.n_kv[t] == 0 || !ok) continue;
+        const int rg = it.tp * 256 + t * 128 + m;
+        const int tok = rg >> lg;
+        const bool valid = tok < it.E;
+        const int64_t orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));
+        ok = mbar_wait(smem_u32(&sm.l_full[t]), done[t] & 1, abortp);
+        if (ok) ok = mbar_wait(smem_u32(&sm.o_full[t]), done[t] & 1, abortp);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const float inv = sm.inv_l[t][done[t] & 1][m];
+        ++done[t];
+        const uint32_t o_addr = lane_base + 256 + t * 128;
+        // A row is 2 * D contiguous bytes, but a warp holds 32 different rows: 16-byte stores from the thread
+        // that owns the row touch 32 cache lines per instruction and half a sector each.  Instead two
+        // neighbouring lanes exchange 32-byte pieces, so that every store instruction writes 64 contiguous
+        // bytes per lane pair, in 32-byte (whole sector) pieces.
+        const int q = lane & 1;
+        char* row_ptr = reinterpret_cast<char*>(a.out + orow_idx * D);
+        // the neighbour's row and whether it exists
+        const uint32_t n_lo = __shfl_xor_sync(0xffffffffu, (uint32_t)reinterpret_cast<uintptr_t>(row_ptr), 1);
+        const uint32_t n_hi = __shfl_xor_sync(0xffffffffu, (uint32_t)(reinterpret_cast<uintptr_t>(row_ptr) >> 32), 1);
+        char* nb_ptr = reinterpret_cast<char*>(((uint64_t)n_hi << 32) | n_lo);
+        const bool nb_valid = __shfl_xor_sync(0xffffffffu, (int)valid, 1) != 0;
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t orow[32];
+          tmem_ld32(o_addr + c * 32, orow);
+          tmem_wait_ld();
+          if (c == D / 32 - 1) {  // all of the row has been read: the next item's PV may overwrite O
+            tc_fence_before_sync();
+            mbar_arrive(smem_u32(&sm.o_empty[t]));
+          }
+          uint32_t pk[16];  // columns [32c, 32c + 32) as bf16 pairs: two pieces of eight words
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const float lo = __uint_as_float(orow[2 * i]) * inv, hi = __uint_as_float(orow[2 * i + 1]) * inv;
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk[i]) : "f"(hi), "f"(lo));
+          }
+          // piece q of the own row is stored by this lane, piece 1-q by the neighbour, and vice versa
+          uint32_t w[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const uint32_t give = q == 0 ? pk[8 + i] : pk[i];
+            w[i] = __shfl_xor_sync(0xffffffffu, give, 1);
+          }
+          // first store: the even lane's row (its own piece 0, and piece 1 handed to the odd lane);
+          // second store: the odd lane's row
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            const bool own = (q == r);
+            if (own ? valid : nb_valid) {
+              char* dst = (own ? row_ptr : nb_ptr) + c * 64 + q * 32;
+              uint32_t d[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i) d[i] = own ? (r == 0 ? pk[i] : pk[8 + i]) : w[i];
+              asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(d[0]), "r"(d[1]), "r"(d[2]), "r"(d[3]),
+                           "r"(d[4]), "r"(d[5]), "r"(d[6]), "r"(d[7])
+                           : "memory");
+            }
+          }
+        }
+      }
+    }
   } else {
     // =============================== softmax warpgroups ======================================
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
-    const int t = (warp - 4) >> 2;                 // query tile of this warpgroup (warps 4-7: tile 0, 8-11: tile 1)
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 192;");
+    const int t = warp >> 2;                       // query tile of this warpgroup (warps 0-3: tile 0, 4-7: tile 1)
     const int w4 = warp & 3;                       // TMEM lane quarter this warp may access
     const int m = w4 * 32 + lane;                  // row inside the tile
     const uint32_t lane_base = tmem + ((uint32_t)(w4 * 32) << 16);
     const uint32_t s_addr = lane_base + t * 128, o_addr = lane_base + 256 + t * 128;
-    const uint32_t bar_s_full = smem_u32(&sm.s_full[t]), bar_o_full = smem_u32(&sm.o_full[t]);
+    const uint32_t bar_s_full = smem_u32(&sm.s_full[t]), bar_l_full = smem_u32(&sm.l_full[t]);
     const uint32_t bar_p_full = smem_u32(&sm.p_full[t]);
     const int G = a.group, lg = a.lg_group, Hq = a.n_q_heads;
-    uint32_t steps = 0, items_done = 0;            // phases of s_full / p_full and of q_full / o_full
+    uint32_t steps = 0, items_done = 0;            // phase of s_full / p_full; items finished (parity of inv_l)
     bool ok = true;
 
     // The item records are read where they are needed (they stay in L1) instead of being carried in registers
@@ -459,7 +629,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       int64_t orow_idx;
       {
         Item it;
-        if (!fetch_item(a, item_index(round), n_total, it)) break;
+        const bool more_items = fetch_item(a, sched_get(round), n_total, it);
+        if (!more_items) break;
+        sched_release(round);
         if (it.ld_tiles == 0) continue;
         n_t = it.n_kv[t];
         if (n_t == 0) continue;
@@ -467,7 +639,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         const int tok = rg >> lg;
         valid = tok < it.E;
         limit = valid ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
-        orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));
+        orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));  // row of the LSE
       }
       float m_run = -INFINITY, l_run = 0.f;
 
@@ -543,41 +715,18 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      // ---- epilogue: O / l -> bf16, LSE
-      ok = mbar_wait(bar_o_full, items_done & 1, abortp);
+      // ---- hand the row to the epilogue warps: 1 / row sum through shared memory; the LSE is written here
+      sm.inv_l[t][items_done & 1][m] = 1.f / l_run;
+      mbar_arrive(bar_l_full);
       ++items_done;
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      tc_fence_after_sync();
-      const float inv = 1.f / l_run;
-#pragma unroll
-      for (int c = 0; c < D / 32; ++c) {
-        uint32_t orow[32];
-        tmem_ld32(o_addr + c * 32, orow);
-        tmem_wait_ld();
-        if (valid) {
-          uint4* dst = reinterpret_cast<uint4*>(a.out + orow_idx * D + c * 32);
-#pragma unroll
-          for (int v4 = 0; v4 < 4; ++v4) {
-            uint32_t w[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const float lo = __uint_as_float(orow[v4 * 8 + 2 * i]) * inv, hi = __uint_as_float(orow[v4 * 8 + 2 * i + 1]) * inv;
-              asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i]) : "f"(hi), "f"(lo));
-            }
-            dst[v4] = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        }
-      }
       if (valid) a.lse[orow_idx] = (m_run + log2f(l_run)) * 0.6931471805599453f;
-      tc_fence_before_sync();
     }
   }
 
   tc_fence_before_sync();
   __syncthreads();
   if (tid == 0 && sm.abort_flag != 0) report(a.pool.status, KV_ERR_TIMEOUT);
-  if (warp == 0) tmem_dealloc(tmem, 512);
+  if (warp == kWarpProducer) tmem_dealloc(tmem, 512);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -626,22 +775,28 @@ static kv_status_t make_q_map(CUtensorMap* map, const void* q, int total_q, int 
   return r == CUDA_SUCCESS ? KV_OK : KV_ERR_INVALID;
 }
 
-template <int D>
-static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int n_items_bound, int cta_cap, cudaStream_t st) {
+// One persistent CTA per SM, fewer if there are fewer items or the caller caps the kernel.
+static kv_status_t tc_grid(int n_items_bound, int cta_cap, int* grid_out) {
   static int sm_count = 0;
   if (sm_count == 0) {
     int dev = 0;
     KV_CUDA_OK(cudaGetDevice(&dev));
     KV_CUDA_OK(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
   }
-  const size_t smem = sizeof(TcSmem<D>) + 1024;
+  int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
+  if (cta_cap > 0 && grid > cta_cap) grid = cta_cap;  // leave the other SMs to work that runs beside this kernel
+  *grid_out = grid;
+  return KV_OK;
+}
+
+template <int D>
+static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid, cudaStream_t st) {
+  const size_t smem = sizeof(TcSmem<D>);
   static bool configured = false;
   if (!configured) {
     KV_CUDA_OK(cudaFuncSetAttribute(attn_extend_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured = true;
   }
-  int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
-  if (cta_cap > 0 && grid > cta_cap) grid = cta_cap;  // leave the other SMs to work that runs beside this kernel
   attn_extend_tc_kernel<D><<<grid, kTcThreads, smem, st>>>(a, q_map);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
@@ -655,7 +810,8 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   const size_t need = extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch, total_q, max_total_len);
   if (workspace == nullptr || workspace_bytes < need) return KV_ERR_WORKSPACE;
   const int G = n_q_heads / p->n_kv_heads;
-  if ((reinterpret_cast<uintptr_t>(q) & 15) != 0) return KV_ERR_INVALID;
+  // Q is read through a tensor map (16-byte base), O is written with 32-byte stores
+  if ((reinterpret_cast<uintptr_t>(q) & 15) != 0 || (reinterpret_cast<uintptr_t>(out) & 31) != 0) return KV_ERR_INVALID;
   CUtensorMap q_map;
   {
     const kv_status_t ms = make_q_map(&q_map, q, total_q, n_q_heads, p->head_dim, G);
@@ -668,8 +824,15 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   const int64_t capacity = item_capacity(n_q_heads, p->n_kv_heads, batch, total_q);
   const int max_tp = (int)(((int64_t)max_extend_len * G + 255) / 256);
   const int max_steps = 2 * ((max_total_len + 127) / 128);
+  const int64_t bound = (int64_t)batch * max_tp * p->n_kv_heads;
+  const int n_bound = bound > (1 << 30) ? (1 << 30) : (int)bound;
+  int grid = 1;
+  {
+    const kv_status_t gs = tc_grid(n_bound, cta_cap, &grid);
+    if (gs != KV_OK) return gs;
+  }
   extend_tc_plan_kernel<<<1, 1024, 0, st>>>(prefix_lens, extend_lens, cu_q, batch, max_tp, lg, max_steps, (int)capacity,
-                                            max_pages, p->d_status, items, n_items);
+                                            max_pages, p->d_status, items, n_items, n_items + 1, grid);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
 
@@ -690,10 +853,9 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   a.lse = lse;
   a.items = items;
   a.n_items = n_items;
-  const int64_t bound = (int64_t)batch * max_tp * p->n_kv_heads;
-  const int n_bound = bound > (1 << 30) ? (1 << 30) : (int)bound;
-  if (p->head_dim == 128) return launch_tc<128>(a, q_map, n_bound, cta_cap, st);
-  return launch_tc<64>(a, q_map, n_bound, cta_cap, st);
+  a.next_item = n_items + 1;
+  if (p->head_dim == 128) return launch_tc<128>(a, q_map, grid, st);
+  return launch_tc<64>(a, q_map, grid, st);
 }
 
 }  // namespace kvattn

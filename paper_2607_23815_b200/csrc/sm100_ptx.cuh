@@ -49,6 +49,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
+// Non-blocking test: has the phase with the given parity completed?
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
 constexpr uint64_t kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait in these kernels
 
 // Waits for the phase with the given parity.  Returns false if `*abort_flag` (shared memory) was
@@ -89,6 +100,12 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const void* tenso
           dst_smem),
       "l"(tensor_map), "r"(x), "r"(y), "r"(z), "r"(bar)
       : "memory");
+}
+
+// Brings the box into L2 only (no shared-memory destination, no completion signal).
+__device__ __forceinline__ void tma_prefetch_3d(const void* tensor_map, int x, int y, int z) {
+  asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(tensor_map), "r"(x), "r"(y), "r"(z)
+               : "memory");
 }
 
 // ---- tensor memory ------------------------------------------------------------------------
