@@ -309,6 +309,8 @@ def extra_measurements(args, dev, peaks, flush):
     steps, warm = max(5, args.steps), 3
     if "reuse" in sections:
         out.update(reuse_vs_recompute(args, dev, peaks, flush))
+    if "fanout" in sections:
+        out.update(fanout_measurement(args, dev, peaks, flush))
     if not sections & {"decode", "append"}:
         if "mixed" in sections:
             out.update(mixed_measurement(args, dev, flush, steps, warm))
@@ -402,6 +404,35 @@ def reuse_vs_recompute(args, dev, peaks, flush):
     return res
 
 
+def fanout_measurement(args, dev, peaks, flush):
+    """Children over a shared parent prefix (32 parents x 17 children, prefix ~2144, suffix ~37): one call that reads
+    the shared pages once per parent against the same children run as independent sequences on aliased block tables."""
+    from paper_2607_23815_b200.workload import FanoutWorkload
+    fw = FanoutWorkload(synth.Geometry(32, 8, 128), device=dev)
+    from paper_2607_23815_b200 import kvattn
+    ms_ind, _ = time_steps(lambda _: fw.independent(), 10, 3, flush, 1)
+    kvattn.kvattn_set_shared_impl(1)   # shared part, own part, merge: three kernels
+    ms_split, _ = time_steps(lambda _: fw.shared(), 10, 3, flush, 1)
+    kvattn.kvattn_set_shared_impl(0)   # the default picks the one-kernel walk for this suffix length
+    ms_sh, _ = time_steps(lambda _: fw.shared(), 10, 3, flush, 1)
+    t_ind, t_sh, t_split = statistics.mean(ms_ind), statistics.mean(ms_sh), statistics.mean(ms_split)
+    d_o = (fw.out.float() - fw.out2.float()).abs().max().item()
+    d_l = (fw.lse - fw.lse2).abs().max().item()
+    fl = fw.flops()
+    res = {"fanout": {
+        "workload": f"{fw.n_parents} parents x {fw.n_children // fw.n_parents} children, Hq=32 Hkv=8 D=128, prefix "
+                    f"{min(fw.parent_lens)}..{max(fw.parent_lens)}, suffix {min(fw.child_lens)}..{max(fw.child_lens)}",
+        "independent_ms": round(t_ind, 4), "shared_ms": round(t_sh, 4), "speedup": round(t_ind / t_sh, 2),
+        "shared_three_kernel_ms": round(t_split, 4),
+        "independent_tflops": round(fl / t_ind / 1e9, 1), "shared_tflops": round(fl / t_sh / 1e9, 1),
+        "shared_frac_of_measured_peak": round(fl / t_sh / 1e9 / peaks["bf16_tflops"], 4),
+        "max_abs_diff_o": d_o, "max_abs_diff_lse": d_l}}
+    fw.close()
+    del fw
+    torch.cuda.empty_cache()
+    return res
+
+
 def mixed_measurement(args, dev, flush, steps, warm):
     """One sem_map -> sem_filter pipeline step: extend set and decode set together."""
     from paper_2607_23815_b200.workload import DeviceWorkload
@@ -475,8 +506,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=HEADLINE, choices=[k for k, v in synth.WORKLOADS.items() if v.n_extend])
     ap.add_argument("--cpu-sample", type=int, default=64, help="tuples in the CPU-oracle sample")
-    ap.add_argument("--sections", default="decode,append,mixed,reuse",
-                    help="extra measurements after the headline: comma list of decode, append, mixed, reuse (or 'none')")
+    ap.add_argument("--sections", default="decode,append,mixed,reuse,fanout",
+                    help="extra measurements after the headline: comma list of decode, append, mixed, reuse, fanout "
+                         "(or 'none')")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle legs (for profiler captures)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup

@@ -168,6 +168,31 @@ kv_status_t attn_extend(kv_pool_t* pool, const void* q, int n_q_heads, const int
                         int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* Extend for children that share a parent's prefix (the dependent tasks a Cartesian product creates
+ * over one parent task, Sections 5.1 and 5.3).  Parent g owns parent_lens[g] tokens in the pages of
+ * parent_tables[g]; its children are the sequences cu_children[g] .. cu_children[g+1]-1.  Child c has
+ * child_lens[c] tokens of its own in the pages of child_tables[c] (kv_append first) and its suffix
+ * token t sees the parent's parent_lens[g] keys followed by its own keys 0..t.  For parent lengths
+ * that are multiples of the page size this is attn_extend with every child's block table = the
+ * parent's pages followed by its own, but the shared pages are read once per parent for all its
+ * children (their query rows are stacked), not once per child.
+ * q/out [dev] bf16 [total_q][n_q_heads][head_dim] (out 32-byte aligned), rows ragged by cu_q
+ * [dev][n_children+1], children of a parent consecutive; lse [dev] fp32 [total_q][n_q_heads];
+ * cu_children [dev][n_parents+1]; parent_tables [dev][n_parents][max_pages_parent]; parent_lens
+ * [dev][n_parents]; child_tables [dev][n_children][max_pages_child]; child_lens [dev][n_children].
+ * Host-side upper bounds: max_child_len >= child_lens[c]; max_parent_rows >= the suffix tokens of
+ * all children of one parent; max_parent_len >= parent_lens[g].  Scratch:
+ * attn_extend_shared_workspace_bytes().  The two partial results of a row (shared part, own part)
+ * are each rounded to bf16 before they are merged. */
+size_t attn_extend_shared_workspace_bytes(const kv_pool_t* pool, int n_q_heads, int n_parents, int n_children,
+                                          int total_q, int max_parent_len);
+kv_status_t attn_extend_shared(kv_pool_t* pool, const void* q, int n_q_heads, const int* cu_q, const int* cu_children,
+                               const int* parent_tables, int max_pages_parent, const int* parent_lens,
+                               const int* child_tables, int max_pages_child, const int* child_lens, int n_parents,
+                               int n_children, int total_q, int max_child_len, int max_parent_rows,
+                               int max_parent_len, float scale, void* out, float* lse, void* workspace,
+                               size_t workspace_bytes, void* stream);
+
 /* Decode ("one token at a time, attending over all previously computed KV", Section 2.1): one query
  * per sequence at position ctx_lens[i]-1 over keys 0..ctx_lens[i]-1 (its own K/V already appended).
  * q/out [dev] bf16 [batch][n_q_heads][head_dim]; lse [dev] fp32 [batch][n_q_heads]; ctx_lens [dev]
@@ -226,6 +251,9 @@ kv_status_t kv_last_async_status(kv_pool_t* pool);
 /* Selects the extend kernel: 0 = automatic, 1 = the small-tile kernel (rows of one KV head read K/V
  * straight from HBM), 2 = the tcgen05 tensor-core kernel.  Process-wide; for tests and benchmarks. */
 kv_status_t kvattn_set_extend_impl(int impl);
+/* Test/tuning hook for attn_extend_shared: 0 = choose by the mean suffix length (default), 1 = three kernels
+ * (shared part, own part, merge), 2 = one kernel that walks the parent's and then the children's tiles. */
+kv_status_t kvattn_set_shared_impl(int impl);
 /* Tuning: inside attn_mixed (both sets present) the persistent extend kernel takes at most n SMs, so that the
  * HBM-bound decode kernel runs beside it on the others instead of after it.  0 = no limit.  Process-wide. */
 kv_status_t kvattn_set_mixed_extend_ctas(int n);

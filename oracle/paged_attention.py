@@ -19,6 +19,10 @@ What it computes, and the passages it restates:
   operator "only prefills the map-specific suffix").  -> ``attn_extend``.
   The suffix token t of a prompt [S | C(t) | I] sits at absolute position
   P + t, sees every prefix key and the suffix keys up to itself.
+* A Cartesian product turns one finished task into several dependent tasks
+  that all reuse the parent's prefix (Section 5.1, "dependent tasks";
+  Section 5.3, the Complete procedure).  -> ``attn_extend_shared``: child c of
+  parent g sees the parent's P_g keys followed by its own suffix so far.
 * Reuse does not change results (Section 1: scheduling "does not change query
   semantics or output accuracy").  So the result has a plain definition,
   softmax(q K^T * scale) V over the visible keys, and this oracle is that
@@ -40,7 +44,8 @@ Pins (tests/test_oracle_pins.py): hand-worked closed form, brute force with an
 independently written evaluation, K == 0 closed form (mean of V, LSE = ln n),
 planted needle, rows of probabilities sum to 1, reuse == from-scratch prefill,
 page-permutation invariance, GQA == MHA on repeated KV heads, decode ==
-extend(E=1), split-and-combine identity, torch's fp64 SDPA as a black box.
+extend(E=1), split-and-combine identity, torch's fp64 SDPA as a black box;
+children sharing a parent == every child on a private copy of the prefix.
 No function here is "parity unpinned".
 """
 from __future__ import annotations
@@ -277,6 +282,42 @@ def attn_extend(pool: PagePool, q_bits, n_q_heads, cu_q, block_tables, prefix_le
             o, l = attention_rows(qf[r0:r0 + E, h, :], kf[:, g, :], vf[:, g, :], visible, scale)
             out[r0:r0 + E, h, :] = o
             lse[r0:r0 + E, h] = l
+    return out, lse
+
+
+def attn_extend_shared(pool: PagePool, q_bits, n_q_heads, cu_q, cu_children, parent_tables, parent_lens,
+                       child_tables, child_lens, scale):
+    """Children of one parent attend over the parent's prefix and their own suffix.
+
+    Parent g holds parent_lens[g] tokens in the pages of parent_tables[g]; its
+    children are cu_children[g] .. cu_children[g+1]-1.  Child c holds
+    child_lens[c] tokens of its own in child_tables[c]; its suffix token t sees
+    the parent's keys 0..P_g-1 and then its own keys 0..t (Section 5.1: the
+    dependent tasks of a Cartesian product reuse the upstream task's prefix).
+    q_bits: uint16 [T_q][Hq][D], child c's rows are cu_q[c] .. cu_q[c+1]-1.
+    Returns float64 O [T_q][Hq][D], LSE [T_q][Hq].
+    """
+    T_q, D = q_bits.shape[0], pool.head_dim
+    G = n_q_heads // pool.n_kv_heads
+    qf = widen(q_bits)
+    out = np.zeros((T_q, n_q_heads, D))
+    lse = np.full((T_q, n_q_heads), -np.inf)
+    for g in range(len(parent_lens)):
+        P = int(parent_lens[g])
+        kp, vp = pool.gather(parent_tables[g], P)
+        for c in range(int(cu_children[g]), int(cu_children[g + 1])):
+            E = int(child_lens[c])
+            if E <= 0:
+                continue
+            kc, vc = pool.gather(child_tables[c], E)
+            kf = widen(np.concatenate([kp, kc], axis=0))     # the child's keys: parent's, then its own
+            vf = widen(np.concatenate([vp, vc], axis=0))
+            r0 = int(cu_q[c])
+            visible = P + np.arange(E) + 1
+            for h in range(n_q_heads):
+                o, l = attention_rows(qf[r0:r0 + E, h, :], kf[:, h // G, :], vf[:, h // G, :], visible, scale)
+                out[r0:r0 + E, h, :] = o
+                lse[r0:r0 + E, h] = l
     return out, lse
 
 

@@ -15,7 +15,19 @@ bool extend_tc_supported(const kv_pool_t* p, int n_q_heads);
 kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
-                             void* workspace, size_t workspace_bytes, int cta_cap, cudaStream_t st);
+                             void* workspace, size_t workspace_bytes, int cta_cap, int mode, const FanArgs* fan,
+                             cudaStream_t st);
+
+size_t extend_shared_workspace_bytes(const kv_pool_t* p, int n_q_heads, int n_parents, int n_children, int total_q,
+                                     int max_parent_len);
+kv_status_t launch_extend_shared(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* cu_children,
+                                 const int* parent_tables, int max_pages_parent, const int* parent_lens,
+                                 const int* child_tables, int max_pages_child, const int* child_lens, int n_parents,
+                                 int n_children, int total_q, int max_child_len, int max_parent_rows, int max_parent_len,
+                                 float scale, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                                 cudaStream_t st);
+
+extern std::atomic<int> g_shared_impl;
 
 static std::atomic<int> g_extend_impl{0};
 static std::atomic<int> g_mixed_extend_ctas{0};  // SMs the extend kernel may take inside attn_mixed (0 = all)
@@ -65,8 +77,8 @@ static kv_status_t extend_impl(kv_pool_t* p, const void* q, int n_q_heads, const
   if (impl == 2 && !tc_ok) return KV_ERR_UNSUPPORTED;
   if (impl == 2 || (impl == 0 && tc_ok)) {
     return launch_extend_tc(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
-                            max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, cta_cap,
-                            (cudaStream_t)stream);
+                            max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, cta_cap, 0,
+                            nullptr, (cudaStream_t)stream);
   }
   return launch_extend_small(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch,
                              max_extend_len, max_total_len, scale, out, lse, (cudaStream_t)stream);
@@ -78,6 +90,42 @@ kv_status_t attn_extend(kv_pool_t* p, const void* q, int n_q_heads, const int* c
                         size_t workspace_bytes, void* stream) {
   return extend_impl(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
                      max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, 0, stream);
+}
+
+size_t attn_extend_shared_workspace_bytes(const kv_pool_t* p, int n_q_heads, int n_parents, int n_children, int total_q,
+                                          int max_parent_len) {
+  if (p == nullptr || n_q_heads <= 0) return 0;
+  return extend_shared_workspace_bytes(p, n_q_heads, n_parents, n_children, total_q, max_parent_len);
+}
+
+kv_status_t attn_extend_shared(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* cu_children,
+                               const int* parent_tables, int max_pages_parent, const int* parent_lens,
+                               const int* child_tables, int max_pages_child, const int* child_lens, int n_parents,
+                               int n_children, int total_q, int max_child_len, int max_parent_rows, int max_parent_len,
+                               float scale, void* out, float* lse, void* workspace, size_t workspace_bytes,
+                               void* stream) {
+  if (p == nullptr || n_parents < 0 || n_children < 0 || total_q < 0 || max_pages_parent < 0 || max_pages_child < 0 ||
+      max_child_len < 0 || max_parent_rows < 0 || max_parent_len < 0)
+    return KV_ERR_INVALID;
+  if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
+  if (n_parents == 0 || n_children == 0 || total_q == 0 || max_child_len == 0) return KV_OK;
+  if (q == nullptr || cu_q == nullptr || cu_children == nullptr || parent_tables == nullptr || parent_lens == nullptr ||
+      child_tables == nullptr || child_lens == nullptr || out == nullptr || lse == nullptr)
+    return KV_ERR_INVALID;
+  if ((((uintptr_t)q) & 15) || (((uintptr_t)out) & 31)) return KV_ERR_INVALID;
+  if (max_parent_len > (int64_t)max_pages_parent * kPageSize || max_child_len > (int64_t)max_pages_child * kPageSize ||
+      max_parent_rows < max_child_len)
+    return KV_ERR_INVALID;
+  if (!(scale > 0.f) || !extend_tc_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
+  return launch_extend_shared(p, q, n_q_heads, cu_q, cu_children, parent_tables, max_pages_parent, parent_lens, child_tables,
+                              max_pages_child, child_lens, n_parents, n_children, total_q, max_child_len, max_parent_rows,
+                              max_parent_len, scale, out, lse, workspace, workspace_bytes, (cudaStream_t)stream);
+}
+
+kv_status_t kvattn_set_shared_impl(int impl) {
+  if (impl < 0 || impl > 2) return KV_ERR_INVALID;
+  g_shared_impl.store(impl);
+  return KV_OK;
 }
 
 kv_status_t kvattn_set_mixed_extend_ctas(int n) {

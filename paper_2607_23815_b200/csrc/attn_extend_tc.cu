@@ -47,6 +47,14 @@ struct TcArgs {
   const int* prefix_lens;
   const int* extend_lens;
   int batch, n_q_heads, group, lg_group;
+  // mode 0: row t of sequence i sees the keys 0 .. P_i + t (extend).
+  // mode 1: every row sees the keys [0, P_i) only.
+  // mode 2 (fan-out): a "sequence" is a parent, its rows are the suffix tokens of its children stacked one
+  //         after the other; a row sees the parent's keys [0, P) and then its own child's keys up to itself.
+  //         The KV steps of an item are the parent's tiles followed by the tiles of every child that has a
+  //         row in the item, each from the child's own pages.
+  int mode;
+  FanArgs fan;
   float scale_log2;
   __nv_bfloat16* out;
   float* lse;
@@ -59,38 +67,60 @@ struct TcArgs {
 // Plan: list the (sequence, tile pair) entries that have rows, heaviest first (counting sort on
 // the number of KV tile steps).  Only the order of execution depends on it, never a result.
 // ------------------------------------------------------------------------------------------
-__device__ __forceinline__ int entry_steps(int P, int E, int tp, int lg) {
-  int steps = 0;
-#pragma unroll
-  for (int t = 0; t < 2; ++t) {
-    const int r_lo = tp * 256 + t * 128;
-    const int tok_lo = r_lo >> lg;
-    if (tok_lo >= E) break;
-    const int tok_hi = min(E - 1, (r_lo + 127) >> lg);
-    steps += (P + tok_hi + 1 + 127) >> 7;
-  }
-  return steps;
-}
-
 // One entry of the plan: everything a CTA needs to know about a (sequence, tile pair), so that the
 // roles read one 32-byte record per item instead of chasing the length arrays.
 struct ItemRec {
   int seq, tp, P, E;
   int row0, n_kv0, n_kv1, kv_end;  // first query row; KV tile steps of the two tiles; keys the item sees at most
+                                   // (fan-out mode: kv_end holds the first child that has a row in the item)
 };
 
-__device__ __forceinline__ ItemRec make_item(int seq, int tp, int P, int E, int row0, int lg, int max_pages) {
+__device__ __forceinline__ ItemRec make_item(int seq, int tp, int P, int E, int row0, int lg, int max_pages, int mode,
+                                             const FanArgs& fan) {
   ItemRec r{seq, tp, P, E, row0, 0, 0, 0};
+  int tok_hi_t[2] = {-1, -1};
 #pragma unroll
   for (int t = 0; t < 2; ++t) {
     const int r_lo = tp * 256 + t * 128;
     const int tok_lo = r_lo >> lg;
     if (tok_lo >= E) break;
     const int tok_hi = min(E - 1, (r_lo + 127) >> lg);
-    (t ? r.n_kv1 : r.n_kv0) = (P + tok_hi + 1 + 127) >> 7;
-    r.kv_end = P + tok_hi + 1;
+    tok_hi_t[t] = tok_hi;
+    const int sees = mode != 0 ? P : P + tok_hi + 1;
+    (t ? r.n_kv1 : r.n_kv0) = (sees + 127) >> 7;
+    r.kv_end = sees;
   }
-  if (P + E > max_pages * kPageSize) r.n_kv0 = r.n_kv1 = 0;  // longer than its block-table row: skipped (reported by the plan)
+  if ((mode != 0 ? P : P + E) > max_pages * kPageSize) r.n_kv0 = r.n_kv1 = 0;  // longer than its block-table row: skipped (reported by the plan)
+  if (mode == 2 && tok_hi_t[0] >= 0) {
+    // children with a row in this item: the first one whose last token lies at or after the item's first token,
+    // then on until a child starts after the item's last token
+    const int c0 = __ldg(fan.cu_children + seq), c1 = __ldg(fan.cu_children + seq + 1);
+    const int tok_lo = (tp * 256) >> lg;
+    int lo = c0, hi = c1;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (__ldg(fan.cu_q + mid + 1) - row0 > tok_lo) hi = mid; else lo = mid + 1;
+    }
+    const int c_first = lo;
+    const int tok_hi_item = max(tok_hi_t[0], tok_hi_t[1]);
+    int extra0 = 0, extra = 0;
+    bool fits = true;
+    for (int c = c_first; c < c1; ++c) {
+      const int start = __ldg(fan.cu_q + c) - row0, len = __ldg(fan.cu_q + c + 1) - __ldg(fan.cu_q + c);
+      if (start > tok_hi_item) break;
+      if (len > fan.max_pages * kPageSize) fits = false;
+      const int st = (len + 127) >> 7;
+      extra += st;
+      if (start <= tok_hi_t[0]) extra0 += st;
+    }
+    r.kv_end = c_first;
+    if (!fits) {
+      r.n_kv0 = r.n_kv1 = 0;
+    } else if (r.n_kv0 > 0 || P == 0) {
+      r.n_kv0 = ((P + 127) >> 7) + extra0;
+      r.n_kv1 = tok_hi_t[1] >= 0 ? ((P + 127) >> 7) + extra : 0;
+    }
+  }
   return r;
 }
 
@@ -98,6 +128,7 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
                                                               const int* __restrict__ extend_lens,
                                                               const int* __restrict__ cu_q, int batch, int max_tp,
                                                               int lg, int max_steps, int capacity, int max_pages,
+                                                              int mode, FanArgs fan,
                                                               int* status, int4* __restrict__ items,
                                                               int* __restrict__ n_items, int* __restrict__ next_item,
                                                               int first_free_item) {
@@ -114,7 +145,9 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
     const int seq = (int)(e / max_tp), tp = (int)(e % max_tp);
     const int P = __ldg(prefix_lens + seq), E = __ldg(extend_lens + seq);
     if (P < 0 || E <= 0) continue;
-    const int steps = entry_steps(P, E, tp, lg);
+    if (((tp * 256) >> lg) >= E) continue;
+    const ItemRec r = make_item(seq, tp, P, E, __ldg(cu_q + seq), lg, max_pages, mode, fan);
+    const int steps = r.n_kv0 + r.n_kv1;
     if (steps > 0) atomicAdd(&hist[key_of(steps)], 1);
   }
   __syncthreads();
@@ -152,12 +185,13 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
     const int seq = (int)(e / max_tp), tp = (int)(e % max_tp);
     const int P = __ldg(prefix_lens + seq), E = __ldg(extend_lens + seq);
     if (P < 0 || E <= 0) continue;
-    const int steps = entry_steps(P, E, tp, lg);
+    if (((tp * 256) >> lg) >= E) continue;
+    const ItemRec r = make_item(seq, tp, P, E, __ldg(cu_q + seq), lg, max_pages, mode, fan);
+    const int steps = r.n_kv0 + r.n_kv1;
+    if (steps == 0 && (mode == 0 || P > 0 || mode == 2)) report(status, KV_ERR_BOUNDS);  // rows exist but the lengths do not fit the tables
     if (steps > 0) {
       const int pos = atomicAdd(&hist[key_of(steps)], 1);
       if (pos < capacity) {
-        const ItemRec r = make_item(seq, tp, P, E, __ldg(cu_q + seq), lg, max_pages);
-        if (r.n_kv0 == 0) report(status, KV_ERR_BOUNDS);
         items[2 * pos] = make_int4(r.seq, r.tp, r.P, r.E);
         items[2 * pos + 1] = make_int4(r.row0, r.n_kv0, r.n_kv1, r.kv_end);
       }
@@ -201,8 +235,41 @@ struct Item {
   int seq, kvh, tp, P, E, row0;
   int n_kv[2];   // KV tile steps of the two query tiles (0 = tile has no rows)
   int ld_tiles;  // KV tiles the producer brings in
-  int kv_end;    // keys the item can see at most
+  int kv_end;    // keys the item can see at most (fan-out mode: the parent's keys)
+  int c_first;   // fan-out mode: first child with a row in the item
 };
+
+// Fan-out mode: position in the children's part of an item's KV steps.
+struct ChildCur {
+  int c, jc;        // child and 128-key tile inside the child's suffix
+  int start, len;   // the child's first token among the parent's stacked rows, and its length
+};
+__device__ __forceinline__ void child_load(const TcArgs& a, int row0, ChildCur& k) {
+  // children without tokens contribute no step
+  int r0 = __ldg(a.fan.cu_q + k.c), r1 = __ldg(a.fan.cu_q + k.c + 1);
+  while (r1 == r0 && k.c + 1 < a.fan.n_children) {
+    ++k.c;
+    r0 = r1;
+    r1 = __ldg(a.fan.cu_q + k.c + 1);
+  }
+  k.start = r0 - row0;
+  k.len = r1 - r0;
+}
+__device__ __forceinline__ void child_first(const TcArgs& a, const Item& it, ChildCur& k) {
+  k.c = it.c_first;
+  k.jc = 0;
+  child_load(a, it.row0, k);
+}
+__device__ __forceinline__ void child_next(const TcArgs& a, const Item& it, ChildCur& k) {
+  if ((k.jc + 1) * 128 < k.len) {
+    ++k.jc;
+  } else if (k.c + 1 < a.fan.n_children) {
+    ++k.c;
+    k.jc = 0;
+    child_load(a, it.row0, k);
+  }
+}
+__device__ __forceinline__ int child_pages(const ChildCur& k) { return min(8, (k.len - k.jc * 128 + 15) >> 4); }
 
 // Item k of the global list: entry k / Hkv of the plan, KV head k % Hkv.  Returns false past the end.
 __device__ __forceinline__ bool fetch_item(const TcArgs& a, int k, int n_total, Item& it) {
@@ -212,6 +279,11 @@ __device__ __forceinline__ bool fetch_item(const TcArgs& a, int k, int n_total, 
   const int4 r0 = __ldg(a.items + 2 * e), r1 = __ldg(a.items + 2 * e + 1);
   it.seq = r0.x; it.tp = r0.y; it.P = r0.z; it.E = r0.w;
   it.row0 = r1.x; it.n_kv[0] = r1.y; it.n_kv[1] = r1.z; it.kv_end = r1.w;
+  it.c_first = 0;
+  if (a.mode == 2) {
+    it.c_first = r1.w;
+    it.kv_end = it.P;
+  }
   it.kvh = k - e * Hkv;
   it.ld_tiles = max(it.n_kv[0], it.n_kv[1]);
   return true;
@@ -334,11 +406,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       if (!ok) break;
       const int* bt = a.block_tables + (int64_t)it.seq * a.max_pages;
       const size_t head_off = (size_t)it.kvh * Cfg::kBlockBytes;
+      const int n_own = a.mode == 2 ? (it.P + 127) >> 7 : it.ld_tiles;  // tiles from the sequence's (parent's) own pages
+      ChildCur cc{0, 0, 0, 0};
       for (int j = 0; j < it.ld_tiles && ok; ++j) {
-        const int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
+        int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
+        const int* src_bt = bt + j * 8;
+        if (j >= n_own) {  // fan-out mode: a tile of a child's own keys
+          if (j == n_own) child_first(a, it, cc); else child_next(a, it, cc);
+          np = child_pages(cc);
+          src_bt = a.fan.tables + (int64_t)cc.c * a.fan.max_pages + cc.jc * 8;
+        }
         int page = 0;
         if (lane < np) {
-          page = __ldg(bt + j * 8 + lane);
+          page = __ldg(src_bt + lane);
           if ((unsigned)page >= (unsigned)a.pool.num_pages) {
             report(a.pool.status, KV_ERR_BOUNDS);
             page = 0;
@@ -422,8 +502,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         }
         if (ok && elect_one_sync()) mma_commit(smem_u32(&sm.kv_empty[stage]));
         __syncwarp();
+        const int n_own = a.mode == 2 ? (it.P + 127) >> 7 : it.ld_tiles;
+        ChildCur cc{0, 0, 0, 0};
         for (int j = 0; j < it.ld_tiles && ok; ++j) {
-          const int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
+          int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
+          if (j >= n_own) {  // fan-out mode: a tile of a child's own keys
+            if (j == n_own) child_first(a, it, cc); else child_next(a, it, cc);
+            np = child_pages(cc);
+          }
           const uint32_t v_stage = loads % Cfg::kStages;
           ok = mbar_wait(smem_u32(&sm.kv_full[v_stage]), (loads / Cfg::kStages) & 1, abortp);
           ++loads;
@@ -627,6 +713,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       int n_t, limit;
       bool valid;
       int64_t orow_idx;
+      // fan-out mode: the steps from n_own on walk the children's own keys; tok_s is this row's token among the
+      // parent's stacked rows (-1: no such row) and (f_row0, f_child) start the walk
+      int n_own, tok_s = -1, f_row0 = 0;
+      ChildCur cc{0, 0, 0, 0};
       {
         Item it;
         const bool more_items = fetch_item(a, sched_get(round), n_total, it);
@@ -638,8 +728,14 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         const int rg = it.tp * 256 + t * 128 + m;
         const int tok = rg >> lg;
         valid = tok < it.E;
-        limit = valid ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
+        limit = valid && a.mode == 0 ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
         orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));  // row of the LSE
+        n_own = a.mode == 2 ? (it.P + 127) >> 7 : n_t;
+        if (a.mode == 2) {
+          tok_s = valid ? tok : -1;
+          f_row0 = it.row0;
+          cc.c = it.c_first;
+        }
       }
       float m_run = -INFINITY, l_run = 0.f;
 
@@ -651,8 +747,24 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         tc_fence_after_sync();
         // One trip to tensor memory: the row's 128 scores are read into registers, reduced to the row
         // maximum, exponentiated in place and written back as bf16 P.
-        const int kv0 = j * 128;
-        const bool ragged = kv0 + 128 > limit;  // diagonal / last tile: keys past the row's limit are hidden
+        // vis: how many of the tile's 128 key columns this row sees (diagonal / last tile: keys past the row's
+        // limit are hidden; fan-out mode: only the row's own child, up to the row's own token)
+        int vis = limit - j * 128;
+        if (j >= n_own) {
+          if (j == n_own) {
+            cc.jc = 0;
+            child_load(a, f_row0, cc);
+          } else if ((cc.jc + 1) * 128 < cc.len) {
+            ++cc.jc;
+          } else if (cc.c + 1 < a.fan.n_children) {
+            ++cc.c;
+            cc.jc = 0;
+            child_load(a, f_row0, cc);
+          }
+          const int t_local = tok_s - cc.start;
+          vis = (tok_s >= 0 && t_local >= 0 && t_local < cc.len) ? t_local + 1 - cc.jc * 128 : 0;
+        }
+        const bool ragged = vis < 128;
         uint32_t sr[4][32];
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld32(s_addr + c * 32, sr[c]);
@@ -662,7 +774,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
           for (int c = 0; c < 4; ++c)
 #pragma unroll
             for (int i = 0; i < 32; ++i)
-              if (kv0 + c * 32 + i >= limit) sr[c][i] = 0xff800000u;  // -inf by select: NaN-safe
+              if (c * 32 + i >= vis) sr[c][i] = 0xff800000u;  // -inf by select: NaN-safe
         }
         float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
@@ -806,7 +918,8 @@ static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid
 kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
-                             void* workspace, size_t workspace_bytes, int cta_cap, cudaStream_t st) {
+                             void* workspace, size_t workspace_bytes, int cta_cap, int mode, const FanArgs* fan,
+                             cudaStream_t st) {
   const size_t need = extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch, total_q, max_total_len);
   if (workspace == nullptr || workspace_bytes < need) return KV_ERR_WORKSPACE;
   const int G = n_q_heads / p->n_kv_heads;
@@ -832,7 +945,8 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
     if (gs != KV_OK) return gs;
   }
   extend_tc_plan_kernel<<<1, 1024, 0, st>>>(prefix_lens, extend_lens, cu_q, batch, max_tp, lg, max_steps, (int)capacity,
-                                            max_pages, p->d_status, items, n_items, n_items + 1, grid);
+                                            max_pages, mode, fan != nullptr ? *fan : FanArgs{}, p->d_status, items, n_items,
+                                            n_items + 1, grid);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
 
@@ -848,6 +962,8 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   a.n_q_heads = n_q_heads;
   a.group = G;
   a.lg_group = lg;
+  a.mode = mode;
+  a.fan = fan != nullptr ? *fan : FanArgs{};
   a.scale_log2 = scale * 1.4426950408889634f;
   a.out = (__nv_bfloat16*)out;
   a.lse = lse;

@@ -39,6 +39,15 @@ __device__ __forceinline__ void report(int* status, int code) {
   if (status != nullptr) atomicCAS(status, 0, code);
 }
 
+// The children of the fan-out mode.
+struct FanArgs {
+  const int* cu_q;         // [n_children + 1]: first row of each child in Q
+  const int* cu_children;  // [n_parents + 1]: children of parent g are cu_children[g] .. cu_children[g+1]-1
+  const int* tables;       // [n_children][max_pages]: the children's own pages
+  int max_pages;
+  int n_children;
+};
+
 extern std::atomic<int64_t> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 

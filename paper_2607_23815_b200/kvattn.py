@@ -61,6 +61,9 @@ _SIGNATURES = {
     "kv_gather": (_I, [_P, _P, _I, _P, _P, _P]),
     "attn_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I, _I]),
     "attn_extend": (_I, [_P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
+    "attn_extend_shared_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I]),
+    "attn_extend_shared": (_I, [_P, _P, _I, _P, _P, _P, _I, _P, _P, _I, _P, _I, _I, _I, _I, _I, _I, _F, _P, _P, _P, _SZ,
+                                _P]),
     "attn_decode": (_I, [_P, _P, _I, _P, _I, _P, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_decode_static": (_I, [_P, _P, _I, _P, _I, _P, _I, _I, _F, _P, _P, _P]),
     "attn_decode_static_scratch_bytes": (_SZ, []),
@@ -68,6 +71,7 @@ _SIGNATURES = {
     "kv_check_batch": (_I, [_P, _P, _I, _P, _I, _P]),
     "kv_last_async_status": (_I, [_P]),
     "kvattn_set_extend_impl": (_I, [_I]),
+    "kvattn_set_shared_impl": (_I, [_I]),
     "kvattn_set_mixed_extend_ctas": (_I, [_I]),
     "kvattn_launch_count": (_I64, []),
 }
@@ -249,6 +253,28 @@ def attn_extend(pool: Pool, q, cu_q, block_tables, prefix_lens, extend_lens, max
                              _dev_ptr(out), _dev_ptr(lse), _dev_ptr(workspace),
                              0 if workspace is None else workspace.numel() * workspace.element_size(),
                              _stream(stream)), "attn_extend")
+
+
+def kvattn_set_shared_impl(impl: int):
+    _check(lib().kvattn_set_shared_impl(impl), "kvattn_set_shared_impl")
+
+
+def attn_extend_shared_workspace_bytes(pool: Pool, n_q_heads, n_parents, n_children, total_q, max_parent_len) -> int:
+    return lib().attn_extend_shared_workspace_bytes(pool.handle, n_q_heads, n_parents, n_children, total_q,
+                                                    max_parent_len)
+
+
+def attn_extend_shared(pool: Pool, q, cu_q, cu_children, parent_tables, parent_lens, child_tables, child_lens,
+                       max_child_len, max_parent_rows, max_parent_len, scale, out, lse, workspace, stream=None):
+    """Children that share their parent's prefix pages (see the header): the shared pages are read once per parent."""
+    _check(lib().attn_extend_shared(pool.handle, _dev_ptr(q), q.shape[1], _dev_ptr(cu_q), _dev_ptr(cu_children),
+                                    _dev_ptr(parent_tables), parent_tables.shape[1], _dev_ptr(parent_lens),
+                                    _dev_ptr(child_tables), child_tables.shape[1], _dev_ptr(child_lens),
+                                    parent_lens.numel(), child_lens.numel(), q.shape[0], max_child_len,
+                                    max_parent_rows, max_parent_len, float(scale), _dev_ptr(out), _dev_ptr(lse),
+                                    _dev_ptr(workspace),
+                                    0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                    _stream(stream)), "attn_extend_shared")
 
 
 def attn_decode(pool: Pool, q, block_tables, ctx_lens, max_ctx_len, scale, out, lse, workspace=None, stream=None):

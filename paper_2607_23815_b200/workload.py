@@ -201,3 +201,80 @@ class DeviceWorkload:
     def close(self):
         torch.cuda.synchronize()
         self.pool.destroy()
+
+
+class FanoutWorkload:
+    """Children that share their parent's prefix pages (the dependent tasks of a Cartesian product, Section 5.1):
+    n_parents parents with a prefix that is a multiple of the page size, n_children children each with a short
+    suffix of its own on private pages.  Stands in for the paper's join workload (17 right-side tuples per
+    contract); lengths are seeded draws around the given centres."""
+
+    def __init__(self, geom: synth.Geometry, n_parents=32, n_children=17, prefix_centre=2144, prefix_spread=224,
+                 suffix_range=(30, 44), seed=260723820, device="cuda"):
+        self.geom, self.device, self.seed = geom, device, seed
+        g, ps = geom, geom.page_size
+        self.parent_lens = [ps * (synth.uniform_int(seed, 201, i, prefix_centre - prefix_spread,
+                                                    prefix_centre + prefix_spread) // ps) for i in range(n_parents)]
+        self.child_lens = [synth.uniform_int(seed, 202, c, suffix_range[0], suffix_range[1])
+                           for c in range(n_parents * n_children)]
+        self.n_parents, self.n_children = n_parents, n_parents * n_children
+        n_pages = sum(L // ps for L in self.parent_lens) + sum(synth.pages_needed(E, ps) for E in self.child_lens)
+        self.pool = kvattn.kv_pool_create(n_pages, ps, g.n_kv_heads, g.head_dim)
+        ids = kvattn.kv_alloc(self.pool, n_pages)
+        placement = [ids[i] for i in synth.page_permutation(seed, n_pages).tolist()]
+        cur = 0
+        self.parent_rows, self.child_rows = [], []
+        for L in self.parent_lens:
+            self.parent_rows.append(placement[cur:cur + L // ps]); cur += L // ps
+        for E in self.child_lens:
+            n = synth.pages_needed(E, ps)
+            self.child_rows.append(placement[cur:cur + n]); cur += n
+        i32 = lambda x: torch.tensor(np.asarray(x), dtype=torch.int32, device=device)
+        self.parent_tables, self.child_tables = i32(synth.block_table(self.parent_rows)), i32(synth.block_table(self.child_rows))
+        # K/V: parents carry uids 0.., children 100000..
+        for rows, lens, uid0, bt in ((self.parent_rows, self.parent_lens, 0, self.parent_tables),
+                                     (self.child_rows, self.child_lens, 100000, self.child_tables)):
+            ks = [synth.normal_bf16(seed, synth.TAG_K, uid0 + i, 0, L, g.n_kv_heads, g.head_dim, device) for i, L in enumerate(lens)]
+            vs = [synth.normal_bf16(seed, synth.TAG_V, uid0 + i, 0, L, g.n_kv_heads, g.head_dim, device) for i, L in enumerate(lens)]
+            kvattn.kv_append(self.pool, torch.cat(ks), torch.cat(vs), i32(np.concatenate([[0], np.cumsum(lens)])),
+                             i32([0] * len(lens)), i32(list(range(len(lens)))), bt)
+        self.q = torch.cat([synth.normal_bf16(seed, synth.TAG_Q, 100000 + c, 0, E, g.n_q_heads, g.head_dim, device)
+                            for c, E in enumerate(self.child_lens)])
+        self.cu_q = i32(np.concatenate([[0], np.cumsum(self.child_lens)]))
+        self.cu_children = i32(np.arange(n_parents + 1) * n_children)
+        self.parent_lens_d, self.child_lens_d = i32(self.parent_lens), i32(self.child_lens)
+        self.max_parent_rows = max(sum(self.child_lens[g0 * n_children:(g0 + 1) * n_children]) for g0 in range(n_parents))
+        self.out = torch.empty_like(self.q)
+        self.lse = torch.empty((self.q.shape[0], g.n_q_heads), dtype=torch.float32, device=device)
+        self.ws_shared = torch.empty(max(256, kvattn.attn_extend_shared_workspace_bytes(
+            self.pool, g.n_q_heads, n_parents, self.n_children, int(self.q.shape[0]), max(self.parent_lens))),
+            dtype=torch.uint8, device=device)
+        # the same children as independent sequences: block table = the parent's pages, then the child's own
+        child_parent = np.repeat(np.arange(n_parents), n_children)
+        self.alias_tables = i32(synth.block_table([self.parent_rows[gp] + self.child_rows[c] for c, gp in enumerate(child_parent)]))
+        self.alias_prefix = i32([self.parent_lens[gp] for gp in child_parent])
+        self.max_total = max(self.parent_lens[gp] + self.child_lens[c] for c, gp in enumerate(child_parent))
+        self.out2, self.lse2 = torch.empty_like(self.q), torch.empty_like(self.lse)
+        self.ws_alias = torch.empty(max(256, kvattn.attn_workspace_bytes(self.pool, g.n_q_heads, self.n_children,
+                                                                         int(self.q.shape[0]), self.max_total, 0, 0)),
+                                    dtype=torch.uint8, device=device)
+        torch.cuda.synchronize()
+
+    def flops(self) -> float:
+        g = self.geom
+        child_parent = np.repeat(np.arange(self.n_parents), self.n_children // self.n_parents)
+        pairs = sum(E * self.parent_lens[gp] + E * (E + 1) // 2 for E, gp in zip(self.child_lens, child_parent))
+        return 4.0 * g.head_dim * g.n_q_heads * pairs
+
+    def shared(self):
+        kvattn.attn_extend_shared(self.pool, self.q, self.cu_q, self.cu_children, self.parent_tables, self.parent_lens_d,
+                                  self.child_tables, self.child_lens_d, max(self.child_lens), self.max_parent_rows,
+                                  max(self.parent_lens), self.geom.scale, self.out, self.lse, self.ws_shared)
+
+    def independent(self):
+        kvattn.attn_extend(self.pool, self.q, self.cu_q, self.alias_tables, self.alias_prefix, self.child_lens_d,
+                           max(self.child_lens), self.max_total, self.geom.scale, self.out2, self.lse2, self.ws_alias)
+
+    def close(self):
+        torch.cuda.synchronize()
+        self.pool.destroy()

@@ -188,6 +188,52 @@ def test_reuse_equals_from_scratch_prefill():
         assert np.max(np.abs(l_reuse - l_full[P:])) < 1e-12
 
 
+def test_children_sharing_a_parent_equal_private_copies_and_brute_force():
+    # Section 5.1: the dependent tasks of a Cartesian product reuse the parent's prefix.  Sharing the
+    # parent's pages must give what every child gets on a private copy of prefix + own suffix, and what
+    # the independently written evaluation gives on the concatenated keys.
+    rng = np.random.default_rng(515)
+    Hkv, Hq, D, ps = 2, 4, 8, 16
+    parent_lens, n_child, child_lens = [37, 16, 0], [3, 2, 1], [5, 1, 9, 17, 2, 4]
+    pool, parent_rows, parent_kv = _build_pool(rng, parent_lens, Hkv, D, ps=ps, num_pages=96)
+    used = {p for row in parent_rows for p in row}
+    free = [p for p in synth.page_permutation(11, 96).tolist() if p not in used]
+    cu_children = np.concatenate([[0], np.cumsum(n_child)])
+    cu_q = np.concatenate([[0], np.cumsum(child_lens)])
+    q = _rand_bits(rng, (int(cu_q[-1]), Hq, D))
+    child_rows, child_kv, private_rows = [], [], []
+    for g in range(len(parent_lens)):
+        for c in range(cu_children[g], cu_children[g + 1]):
+            E = child_lens[c]
+            k, v = _rand_bits(rng, (E, Hkv, D)), _rand_bits(rng, (E, Hkv, D))
+            n = synth.pages_needed(E, ps)
+            pages, free = free[:n], free[n:]
+            pool.append(pages, 0, k, v)
+            child_rows.append(pages)
+            child_kv.append((k, v))
+            # the private copy: parent's tokens and the child's on pages of its own
+            n2 = synth.pages_needed(parent_lens[g] + E, ps)
+            priv, free = free[:n2], free[n2:]
+            pool.append(priv, 0, np.concatenate([parent_kv[g][0], k]), np.concatenate([parent_kv[g][1], v]))
+            private_rows.append(priv)
+    scale = 0.3
+    o, lse = orc.attn_extend_shared(pool, q, Hq, cu_q, cu_children, synth.block_table(parent_rows), parent_lens,
+                                    synth.block_table(child_rows), child_lens, scale)
+    child_parent = np.repeat(np.arange(len(parent_lens)), n_child)
+    o2, lse2 = orc.attn_extend(pool, q, Hq, cu_q, synth.block_table(private_rows),
+                               [parent_lens[g] for g in child_parent], child_lens, scale)
+    assert np.max(np.abs(o - o2)) < 1e-12 and np.max(np.abs(lse - lse2)) < 1e-12
+    for c, g in enumerate(child_parent):
+        P, E = parent_lens[g], child_lens[c]
+        keys = orc.widen(np.concatenate([parent_kv[g][0], child_kv[c][0]]))
+        vals = orc.widen(np.concatenate([parent_kv[g][1], child_kv[c][1]]))
+        for h in range(Hq):
+            ob, lb = _brute(orc.widen(q[cu_q[c]:cu_q[c + 1], h]).tolist(), keys[:, h // 2].tolist(),
+                            vals[:, h // 2].tolist(), [P + t + 1 for t in range(E)], scale)
+            assert np.max(np.abs(o[cu_q[c]:cu_q[c + 1], h] - ob)) < 1e-12
+            assert np.max(np.abs(lse[cu_q[c]:cu_q[c + 1], h] - lb)) < 1e-12
+
+
 def test_page_permutation_invariance_is_bit_exact():
     rng = np.random.default_rng(21)
     lens = [40, 17, 64, 1]
