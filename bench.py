@@ -418,6 +418,9 @@ def fanout_measurement(args, dev, peaks, flush):
     t_ind, t_sh, t_split = statistics.mean(ms_ind), statistics.mean(ms_sh), statistics.mean(ms_split)
     d_o = (fw.out.float() - fw.out2.float()).abs().max().item()
     d_l = (fw.lse - fw.lse2).abs().max().item()
+    st = kvattn.kv_last_async_status(fw.pool)
+    if st != kvattn.KV_OK:
+        raise RuntimeError(f"fan-out section: device status {st} (a kernel reported an error)")
     fl = fw.flops()
     res = {"fanout": {
         "workload": f"{fw.n_parents} parents x {fw.n_children // fw.n_parents} children, Hq=32 Hkv=8 D=128, prefix "

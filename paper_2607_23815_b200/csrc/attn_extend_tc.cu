@@ -827,7 +827,15 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
-      // ---- hand the row to the epilogue warps: 1 / row sum through shared memory; the LSE is written here
+      // ---- hand the row to the epilogue warps: 1 / row sum through shared memory; the LSE is written here.
+      // The softmax of an item needs only S, so with one-step items it could finish two items before the
+      // epilogue warps have looked at the first: a barrier must not get two phases ahead of its waiters, so
+      // this hand-over waits until the previous item's rows of this tile have been read out.
+      if (items_done > 0) {
+        ok = mbar_wait(smem_u32(&sm.o_empty[t]), (items_done - 1) & 1, abortp);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+      }
       sm.inv_l[t][items_done & 1][m] = 1.f / l_run;
       mbar_arrive(bar_l_full);
       ++items_done;

@@ -199,8 +199,12 @@ class DeviceWorkload:
         return synth.bf16_bits(k), synth.bf16_bits(v)
 
     def close(self):
+        """Destroys the pool; raises if a kernel recorded an error (bounds, a wait that gave up) while it lived."""
         torch.cuda.synchronize()
+        status = kvattn.kv_last_async_status(self.pool)
         self.pool.destroy()
+        if status != kvattn.KV_OK:
+            raise kvattn.KvError(status, "device status at close")
 
 
 class FanoutWorkload:
@@ -276,5 +280,9 @@ class FanoutWorkload:
                            max(self.child_lens), self.max_total, self.geom.scale, self.out2, self.lse2, self.ws_alias)
 
     def close(self):
+        """Destroys the pool; raises if a kernel recorded an error (bounds, a wait that gave up) while it lived."""
         torch.cuda.synchronize()
+        status = kvattn.kv_last_async_status(self.pool)
         self.pool.destroy()
+        if status != kvattn.KV_OK:
+            raise kvattn.KvError(status, "device status at close")

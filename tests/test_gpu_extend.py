@@ -114,3 +114,27 @@ def test_extend_bit_determinism_and_placement_invariance(impl):
         dp.close()
     for o in outs[1:]:
         assert np.array_equal(outs[0]["o_bits"], o["o_bits"]) and np.array_equal(outs[0]["lse_raw"], o["lse_raw"])
+
+
+def test_many_one_step_items_on_the_tensor_core_kernel():
+    # Hundreds of sequences whose keys fit one 128-key tile: every work item is a single softmax step, so the
+    # roles of the kernel run as far ahead of each other as their hand-overs allow.  Repeated, because the
+    # failure this guards against (a hand-over barrier two phases ahead of its waiters) depended on timing.
+    geom = synth.Geometry(32, 8, 128)
+    _skip_if_no_tc(2, geom)
+    rng = np.random.default_rng(77)
+    n = 300
+    E = rng.integers(30, 45, size=n).tolist()
+    P = [0] * n
+    dp = DualPool(geom, 3 * n + 8, seed=277)
+    b = Batch(dp, E)
+    b.write([(i, 0, E[i]) for i in range(n)])
+    for rep in range(6):
+        res = run_extend(dp, b, P, E, impl=2, oracle=(rep == 0))
+        assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+        if rep == 0:
+            assert_close(res, "one-step items")
+            first = res["o_bits"].copy()
+        else:
+            assert np.array_equal(res["o_bits"], first)
+    dp.close()
