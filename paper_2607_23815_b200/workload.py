@@ -210,8 +210,8 @@ class DeviceWorkload:
 class FanoutWorkload:
     """Children that share their parent's prefix pages (the dependent tasks of a Cartesian product, Section 5.1):
     n_parents parents with a prefix that is a multiple of the page size, n_children children each with a short
-    suffix of its own on private pages.  Stands in for the paper's join workload (17 right-side tuples per
-    contract); lengths are seeded draws around the given centres."""
+    suffix of its own on private pages.  Stands in for the paper's join workload (contracts of about 2,145 tokens
+    with 17 right-side tuples each, Section 7.3); lengths are seeded draws around the given centres."""
 
     def __init__(self, geom: synth.Geometry, n_parents=32, n_children=17, prefix_centre=2144, prefix_spread=224,
                  suffix_range=(30, 44), seed=260723820, device="cuda"):
