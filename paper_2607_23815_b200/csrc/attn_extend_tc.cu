@@ -3,7 +3,9 @@
 // Work item = (sequence, KV head, pair of 128-row query tiles).  The rows of a tile are the
 // (suffix token, query head of the KV head's group) pairs, token-major, so the G query heads that
 // share a KV head share every K/V tile that is brought on chip (GQA) and the causal diagonal is
-// only 128/G tokens wide.  One persistent CTA per SM walks a cost-sorted item list.
+// only 128/G tokens wide.  One persistent CTA per SM; the items are sorted by cost and taken heaviest
+// first from a global counter, so a CTA that finishes early simply takes more.
+// Besides extend, the kernel has a prefix-only mode and a fan-out mode (see TcArgs::mode).
 //
 // Roles (warp-specialised, 16 warps):
 //   warps 0-3   softmax of query tile 0: one thread per row (= TMEM lane): masks, running max and
