@@ -107,12 +107,25 @@ __global__ void __launch_bounds__(256, 1) attn_small_kernel(SmallArgs a, int64_t
   if (item >= total_items) return;
 
   const int Hkv = a.pool.n_kv_heads, G = a.group, Hq = a.n_q_heads;
-  const int chunk = (int)(item % a.max_chunks);
-  int64_t rest = item / a.max_chunks;
-  const int rt = (int)(rest % a.max_row_tiles);
-  rest /= a.max_row_tiles;
-  const int kvh = (int)(rest % Hkv);
-  const int seq = (int)(rest / Hkv);
+  int chunk, rt, kvh, seq;
+  if (EXTEND) {
+    chunk = (int)(item % a.max_chunks);
+    int64_t rest = item / a.max_chunks;
+    rt = (int)(rest % a.max_row_tiles);
+    rest /= a.max_row_tiles;
+    kvh = (int)(rest % Hkv);
+    seq = (int)(rest / Hkv);
+  } else {
+    // Decode: the chunk index is the slowest dimension.  Blocks start in index order, so every sequence's first
+    // (full) chunks go first and the last, partly filled or empty chunks of the longer sequences go last: the
+    // kernel's tail, when the SMs run out of work one by one, is made of the smallest pieces.
+    const int64_t per_chunk = (int64_t)a.batch * Hkv;
+    chunk = (int)(item / per_chunk);
+    const int rest = (int)(item % per_chunk);
+    rt = 0;
+    kvh = rest % Hkv;
+    seq = rest / Hkv;
+  }
 
   int P = 0, E = 1, L, row0;
   if (EXTEND) {
