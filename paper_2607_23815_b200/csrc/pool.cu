@@ -21,16 +21,15 @@ __global__ void __launch_bounds__(256) append_kernel(PoolView pool, const uint4*
                                                      const int* __restrict__ seg_row,
                                                      const int* __restrict__ block_tables, int max_pages,
                                                      int n_segments, int total_new) {
+  // One warp per token: the token's segment, position and page are looked up once, then the lanes copy the
+  // token's 16-byte chunks (n_kv_heads * head_dim / 8 of them), all loads of a token in flight before its stores.
   const int chunks_per_row = pool.head_dim >> 3;               // 16-byte chunks per (token, head)
   const int chunks_per_token = pool.n_kv_heads * chunks_per_row;
-  const int64_t total = (int64_t)total_new * chunks_per_token;
   const size_t blk = block_bytes(pool.head_dim);
-  for (int64_t idx = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-       idx += (int64_t)gridDim.x * blockDim.x) {
-    const int token = (int)(idx / chunks_per_token);
-    const int rem = (int)(idx - (int64_t)token * chunks_per_token);
-    const int head = rem / chunks_per_row;
-    const int dchunk = rem - head * chunks_per_row;
+  const int lane = threadIdx.x & 31;
+  const int warps = (gridDim.x * blockDim.x) >> 5;
+  constexpr int kMaxPerLane = 8;                               // chunks a lane holds at once (256 chunks per pass)
+  for (int token = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; token < total_new; token += warps) {
     // segment of this token: last s with cu_new[s] <= token
     int lo = 0, hi = n_segments;
     while (hi - lo > 1) {
@@ -38,29 +37,49 @@ __global__ void __launch_bounds__(256) append_kernel(PoolView pool, const uint4*
       if (__ldg(cu_new + mid) <= token) lo = mid; else hi = mid;
     }
     const int seg = lo;
-    const int seg_begin = __ldg(cu_new + seg);
-    if (token >= __ldg(cu_new + seg + 1)) continue;            // cu_new not covering this row: skip
+    const int seg_begin = __ldg(cu_new + seg), seg_end = __ldg(cu_new + seg + 1);
+    if (token >= seg_end) continue;                            // cu_new not covering this row: skip
     const int pos = __ldg(start_pos + seg) + (token - seg_begin);
     const int row = seg_row ? __ldg(seg_row + seg) : seg;
     const int blk_idx = pos >> 4;
     if (pos < 0 || blk_idx >= max_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
     const int page = __ldg(block_tables + (int64_t)row * max_pages + blk_idx);
     if (page < 0 || page >= pool.num_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
-    const size_t off = ((size_t)page * pool.n_kv_heads + head) * blk + chunk_offset_bytes(pos & 15, dchunk, pool.head_dim);
-    const uint4 kk = __ldg(k_new + idx);
-    const uint4 vv = __ldg(v_new + idx);
-    *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + off) = kk;
-    *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + off) = vv;
-    // The segment's last token also clears the slots behind it in its page.  Slots past a sequence's
-    // end therefore never hold NaN/Inf bit patterns, which the tensor-core kernel relies on: it
-    // multiplies those V rows by probabilities that are exactly 0.
-    if (token + 1 == __ldg(cu_new + seg + 1)) {
-      const size_t blk_off = ((size_t)page * pool.n_kv_heads + head) * blk;
-      const uint4 z = make_uint4(0, 0, 0, 0);
-      for (int slot = (pos & 15) + 1; slot < kPageSize; ++slot) {
-        const size_t o2 = blk_off + chunk_offset_bytes(slot, dchunk, pool.head_dim);
-        *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + o2) = z;
-        *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + o2) = z;
+    const size_t page_off = (size_t)page * pool.n_kv_heads * blk;
+    const uint4* ksrc = k_new + (int64_t)token * chunks_per_token;
+    const uint4* vsrc = v_new + (int64_t)token * chunks_per_token;
+    const bool last = token + 1 == seg_end;
+    for (int c0 = 0; c0 < chunks_per_token; c0 += 32 * kMaxPerLane) {
+      uint4 kk[kMaxPerLane], vv[kMaxPerLane];
+#pragma unroll
+      for (int i = 0; i < kMaxPerLane; ++i) {
+        const int c = c0 + i * 32 + lane;
+        if (c < chunks_per_token) {
+          kk[i] = __ldg(ksrc + c);
+          vv[i] = __ldg(vsrc + c);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kMaxPerLane; ++i) {
+        const int c = c0 + i * 32 + lane;
+        if (c < chunks_per_token) {
+          const int head = c / chunks_per_row, dchunk = c - head * chunks_per_row;
+          const size_t blk_off = page_off + (size_t)head * blk;
+          const size_t off = blk_off + chunk_offset_bytes(pos & 15, dchunk, pool.head_dim);
+          *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + off) = kk[i];
+          *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + off) = vv[i];
+          // The segment's last token also clears the slots behind it in its page.  Slots past a sequence's
+          // end therefore never hold NaN/Inf bit patterns, which the tensor-core kernel relies on: it
+          // multiplies those V rows by probabilities that are exactly 0.
+          if (last) {
+            const uint4 z = make_uint4(0, 0, 0, 0);
+            for (int slot = (pos & 15) + 1; slot < kPageSize; ++slot) {
+              const size_t o2 = blk_off + chunk_offset_bytes(slot, dchunk, pool.head_dim);
+              *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + o2) = z;
+              *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + o2) = z;
+            }
+          }
+        }
       }
     }
   }
@@ -405,8 +424,7 @@ kv_status_t kv_append(kv_pool_t* p, const void* k_new, const void* v_new, const 
   if (k_new == nullptr || v_new == nullptr || cu_new == nullptr || start_pos == nullptr || block_tables == nullptr)
     return KV_ERR_INVALID;
   if ((((uintptr_t)k_new) | ((uintptr_t)v_new)) & 15) return KV_ERR_INVALID;
-  const int64_t chunks = (int64_t)total_new * p->n_kv_heads * (p->head_dim >> 3);
-  append_kernel<<<grid_for(chunks, 256), 256, 0, (cudaStream_t)stream>>>(
+  append_kernel<<<grid_for((int64_t)total_new * 32, 256), 256, 0, (cudaStream_t)stream>>>(  // one warp per token
       p->view(), (const uint4*)k_new, (const uint4*)v_new, cu_new, start_pos, seg_row, block_tables, max_pages,
       n_segments, total_new);
   count_launch();
