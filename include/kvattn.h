@@ -172,10 +172,11 @@ kv_status_t attn_extend(kv_pool_t* pool, const void* q, int n_q_heads, const int
  * over one parent task, Sections 5.1 and 5.3).  Parent g owns parent_lens[g] tokens in the pages of
  * parent_tables[g]; its children are the sequences cu_children[g] .. cu_children[g+1]-1.  Child c has
  * child_lens[c] tokens of its own in the pages of child_tables[c] (kv_append first) and its suffix
- * token t sees the parent's parent_lens[g] keys followed by its own keys 0..t.  For parent lengths
- * that are multiples of the page size this is attn_extend with every child's block table = the
- * parent's pages followed by its own, but the shared pages are read once per parent for all its
- * children (their query rows are stacked), not once per child.
+ * token t sees the parent's parent_lens[g] keys followed by its own keys 0..t.  (For parent lengths
+ * that are multiples of the page size this equals attn_extend with every child's block table = the
+ * parent's pages followed by its own; other parent lengths are fine here, the children's keys never
+ * share a page with the parent's.)  The shared pages are read once per parent for all its children
+ * (their query rows are stacked), not once per child.
  * q/out [dev] bf16 [total_q][n_q_heads][head_dim] (out 32-byte aligned), rows ragged by cu_q
  * [dev][n_children+1], children of a parent consecutive; lse [dev] fp32 [total_q][n_q_heads];
  * cu_children [dev][n_parents+1]; parent_tables [dev][n_parents][max_pages_parent]; parent_lens

@@ -84,6 +84,14 @@ def test_shared_prefix_children_match_the_oracle(impl, hq, hkv, d):
 
 
 @pytest.mark.parametrize("impl", IMPLS)
+def test_parent_lengths_need_not_be_page_multiples(impl):
+    # the children's keys come from their own pages, so the parent may end anywhere inside a page
+    geom = synth.Geometry(32, 8, 128)
+    res = _run_shared(geom, [37, 301, 129], [2, 3, 1], [40, 7, 33, 64, 1, 200], seed=931, also_aliased=False, impl=impl)
+    assert_close(res, f"ragged parents impl{impl}")
+
+
+@pytest.mark.parametrize("impl", IMPLS)
 def test_many_short_children_per_tile(impl):
     # suffixes of 1..6 tokens: dozens of children share one query tile, some of them empty
     geom = synth.Geometry(8, 2, 128)
