@@ -183,8 +183,13 @@ kv_status_t attn_extend(kv_pool_t* pool, const void* q, int n_q_heads, const int
  * [dev][n_parents]; child_tables [dev][n_children][max_pages_child]; child_lens [dev][n_children].
  * Host-side upper bounds: max_child_len >= child_lens[c]; max_parent_rows >= the suffix tokens of
  * all children of one parent; max_parent_len >= parent_lens[g].  Scratch:
- * attn_extend_shared_workspace_bytes().  The two partial results of a row (shared part, own part)
- * are each rounded to bf16 before they are merged. */
+ * attn_extend_shared_workspace_bytes().  Errors: KV_ERR_INVALID (NULL pointers, misaligned q/out, bounds
+ * that do not fit the tables), KV_ERR_UNSUPPORTED (head geometry outside the set above, head_dim other
+ * than 64/128, scale <= 0), KV_ERR_WORKSPACE; a table entry or length outside the pool is skipped on
+ * the device and recorded as KV_ERR_BOUNDS (kv_last_async_status).  Nothing is allocated or retained.
+ * With kvattn_set_shared_impl(1) the two partial results of a row (shared part, own part) are each
+ * rounded to bf16 before they are merged; the default for suffixes of 16 tokens and more on average
+ * accumulates both in one fp32 accumulator. */
 size_t attn_extend_shared_workspace_bytes(const kv_pool_t* pool, int n_q_heads, int n_parents, int n_children,
                                           int total_q, int max_parent_len);
 kv_status_t attn_extend_shared(kv_pool_t* pool, const void* q, int n_q_heads, const int* cu_q, const int* cu_children,
