@@ -518,7 +518,10 @@ def run_reference(args):
     w = synth.WORKLOADS[args.workload]
     g = w.geom
     ext, _ = synth.draw_lengths(w)
-    n_s = min(args.cpu_sample, 16, len(ext))               # about a second of host work per step
+    # The sample shrinks with the number of steps asked for, so that the whole run stays near two minutes: a tuple
+    # of this workload costs the oracle about 0.12 s on 8-16 host threads.
+    per_step_budget_s = 150.0 / max(1, args.steps + args.warmup)
+    n_s = max(1, min(args.cpu_sample, 16, len(ext), int(per_step_budget_s / 0.12)))
     P, E = [p for p, _ in ext[:n_s]], [e for _, e in ext[:n_s]]
     pages = sum(synth.pages_needed(p + e, g.page_size) for p, e in zip(P, E))
     host = orc.PagePool(pages, g.page_size, g.n_kv_heads, g.head_dim)
