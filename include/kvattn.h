@@ -168,6 +168,25 @@ kv_status_t attn_extend(kv_pool_t* pool, const void* q, int n_q_heads, const int
                         int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* One pipeline step from host memory: the call for a caller whose suffix Q/K/V, lengths and block tables live
+ * in host buffers (pinned, if the call is to return before the copies are done).  On the given stream it
+ * copies the inputs into `staging` [dev], appends the suffix K/V rows of sequence i at positions
+ * prefix_lens[i].. of its pages (kv_append), runs attn_extend, and copies O and LSE back into out / lse
+ * [host].  All array arguments except staging are HOST pointers with the shapes of kv_append / attn_extend;
+ * staging [dev, 256-byte aligned] holds attn_extend_host_staging_bytes() bytes; it and the host buffers belong
+ * to the call until the stream has passed it.  The copies run on copy streams of the pool, ordered against the
+ * kernels (on `stream`) by events, and the stream waits for the copy out; with two staging areas used in turn
+ * one step's copies overlap its neighbour's kernels.  The copy in starts at once: the host inputs must be
+ * final when the call is made.  At most four staging areas are tracked at a time.  Errors as for kv_append and attn_extend, KV_ERR_WORKSPACE for a staging area that is too
+ * small.  (In the paper the requests reach the engine from host-side operators, Section 3; the paper has
+ * no counterpart of this exact call.) */
+size_t attn_extend_host_staging_bytes(const kv_pool_t* pool, int n_q_heads, int batch, int total_q, int max_pages,
+                                      int max_total_len);
+kv_status_t attn_extend_host(kv_pool_t* pool, const void* q, const void* k_new, const void* v_new, int n_q_heads,
+                             const int* cu_q, const int* block_tables, int max_pages, const int* prefix_lens,
+                             const int* extend_lens, int batch, int total_q, int max_extend_len, int max_total_len,
+                             float scale, void* out, float* lse, void* staging, size_t staging_bytes, void* stream);
+
 /* Extend for children that share a parent's prefix (the dependent tasks a Cartesian product creates
  * over one parent task, Sections 5.1 and 5.3).  Parent g owns parent_lens[g] tokens in the pages of
  * parent_tables[g]; its children are the sequences cu_children[g] .. cu_children[g+1]-1.  Child c has

@@ -122,6 +122,103 @@ kv_status_t attn_extend_shared(kv_pool_t* p, const void* q, int n_q_heads, const
                               max_parent_len, scale, out, lse, workspace, workspace_bytes, (cudaStream_t)stream);
 }
 
+// ---- one call from host buffers ---------------------------------------------------------------
+// Layout of the staging area: the device copies of the inputs and results, each 256-byte aligned, followed by the
+// attention workspace.
+namespace {
+struct HostStepLayout {
+  size_t q, k, v, cu, bt, pl, el, out, lse, ws, total;
+};
+HostStepLayout host_step_layout(const kv_pool_t* p, int n_q_heads, int batch, int total_q, int max_pages, int max_total_len) {
+  HostStepLayout L{};
+  const size_t D = (size_t)p->head_dim;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { const size_t at = o; o += align256(bytes); return at; };
+  L.q = take((size_t)total_q * n_q_heads * D * 2);
+  L.k = take((size_t)total_q * p->n_kv_heads * D * 2);
+  L.v = take((size_t)total_q * p->n_kv_heads * D * 2);
+  L.cu = take(sizeof(int) * ((size_t)batch + 1));
+  L.bt = take(sizeof(int) * (size_t)batch * max_pages);
+  L.pl = take(sizeof(int) * (size_t)batch);
+  L.el = take(sizeof(int) * (size_t)batch);
+  L.out = take((size_t)total_q * n_q_heads * D * 2);
+  L.lse = take((size_t)total_q * n_q_heads * 4);
+  L.ws = o;
+  L.total = o + attn_workspace_bytes(p, n_q_heads, batch, total_q, max_total_len, 0, 0);
+  return L;
+}
+}  // namespace
+
+size_t attn_extend_host_staging_bytes(const kv_pool_t* p, int n_q_heads, int batch, int total_q, int max_pages,
+                                      int max_total_len) {
+  if (p == nullptr || n_q_heads <= 0 || batch <= 0 || total_q <= 0 || max_pages <= 0) return 0;
+  return host_step_layout(p, n_q_heads, batch, total_q, max_pages, max_total_len).total;
+}
+
+kv_status_t attn_extend_host(kv_pool_t* p, const void* q, const void* k_new, const void* v_new, int n_q_heads,
+                             const int* cu_q, const int* block_tables, int max_pages, const int* prefix_lens,
+                             const int* extend_lens, int batch, int total_q, int max_extend_len, int max_total_len,
+                             float scale, void* out, float* lse, void* staging, size_t staging_bytes, void* stream) {
+  if (p == nullptr || batch < 0 || total_q < 0 || max_pages < 0) return KV_ERR_INVALID;
+  if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
+  if (batch == 0 || total_q == 0) return KV_OK;
+  if (q == nullptr || k_new == nullptr || v_new == nullptr || cu_q == nullptr || block_tables == nullptr ||
+      prefix_lens == nullptr || extend_lens == nullptr || out == nullptr || lse == nullptr || staging == nullptr)
+    return KV_ERR_INVALID;
+  if (((uintptr_t)staging) & 255) return KV_ERR_INVALID;
+  const HostStepLayout L = host_step_layout(p, n_q_heads, batch, total_q, max_pages, max_total_len);
+  if (staging_bytes < L.total) return KV_ERR_WORKSPACE;
+  cudaStream_t st = (cudaStream_t)stream;
+  char* d = reinterpret_cast<char*>(staging);
+  const size_t D = (size_t)p->head_dim;
+  const size_t q_bytes = (size_t)total_q * n_q_heads * D * 2, kv_bytes = (size_t)total_q * p->n_kv_heads * D * 2;
+  // The copies run on the pool's own copy streams: a stream that carries copies in both directions and kernels
+  // serialises them, which costs a third of the throughput of back-to-back steps (measured).  Per staging area:
+  // copy in after the kernels that last used it; kernels (caller's stream) after the copy in; copy out after the
+  // kernels; the caller's stream waits for the copy out, so it still orders everything the caller does next.
+  kv_pool::HostSlot* hs = nullptr;
+  {
+    std::lock_guard<std::mutex> g(p->mu);
+    for (auto& c : p->host_slots)
+      if (c.staging == staging) hs = &c;
+    if (hs == nullptr) {
+      hs = &p->host_slots[p->host_slot_next];
+      p->host_slot_next = (p->host_slot_next + 1) % kv_pool::kHostSlots;
+      // the slot's previous staging area is forgotten: wait for what was still using its events
+      if (hs->staging != nullptr) KV_CUDA_OK(cudaEventSynchronize(hs->out));
+      hs->staging = staging;
+    }
+  }
+  KV_CUDA_OK(cudaStreamWaitEvent(p->h2d_stream, hs->ran, 0));  // (a never-recorded event counts as complete)
+  KV_CUDA_OK(cudaMemcpyAsync(d + L.k, k_new, kv_bytes, cudaMemcpyHostToDevice, p->h2d_stream));
+  KV_CUDA_OK(cudaMemcpyAsync(d + L.v, v_new, kv_bytes, cudaMemcpyHostToDevice, p->h2d_stream));
+  KV_CUDA_OK(cudaMemcpyAsync(d + L.q, q, q_bytes, cudaMemcpyHostToDevice, p->h2d_stream));
+  KV_CUDA_OK(cudaMemcpyAsync(d + L.cu, cu_q, sizeof(int) * ((size_t)batch + 1), cudaMemcpyHostToDevice, p->h2d_stream));
+  KV_CUDA_OK(cudaMemcpyAsync(d + L.bt, block_tables, sizeof(int) * (size_t)batch * max_pages, cudaMemcpyHostToDevice,
+                             p->h2d_stream));
+  KV_CUDA_OK(cudaMemcpyAsync(d + L.pl, prefix_lens, sizeof(int) * (size_t)batch, cudaMemcpyHostToDevice, p->h2d_stream));
+  KV_CUDA_OK(cudaMemcpyAsync(d + L.el, extend_lens, sizeof(int) * (size_t)batch, cudaMemcpyHostToDevice, p->h2d_stream));
+  KV_CUDA_OK(cudaEventRecord(hs->in, p->h2d_stream));
+  KV_CUDA_OK(cudaStreamWaitEvent(st, hs->in, 0));
+  const int* d_cu = reinterpret_cast<const int*>(d + L.cu);
+  const int* d_bt = reinterpret_cast<const int*>(d + L.bt);
+  const int* d_pl = reinterpret_cast<const int*>(d + L.pl);
+  const int* d_el = reinterpret_cast<const int*>(d + L.el);
+  // the suffix K/V rows of sequence i go to positions prefix_lens[i] .. of its pages, then the suffix attends
+  kv_status_t s = kv_append(p, d + L.k, d + L.v, d_cu, d_pl, nullptr, d_bt, max_pages, batch, total_q, stream);
+  if (s == KV_OK)
+    s = attn_extend(p, d + L.q, n_q_heads, d_cu, d_bt, max_pages, d_pl, d_el, batch, total_q, max_extend_len,
+                    max_total_len, scale, d + L.out, reinterpret_cast<float*>(d + L.lse), d + L.ws, L.total - L.ws, stream);
+  KV_CUDA_OK(cudaEventRecord(hs->ran, st));
+  if (s != KV_OK) return s;
+  KV_CUDA_OK(cudaStreamWaitEvent(p->d2h_stream, hs->ran, 0));
+  KV_CUDA_OK(cudaMemcpyAsync(out, d + L.out, q_bytes, cudaMemcpyDeviceToHost, p->d2h_stream));
+  KV_CUDA_OK(cudaMemcpyAsync(lse, d + L.lse, (size_t)total_q * n_q_heads * 4, cudaMemcpyDeviceToHost, p->d2h_stream));
+  KV_CUDA_OK(cudaEventRecord(hs->out, p->d2h_stream));
+  KV_CUDA_OK(cudaStreamWaitEvent(st, hs->out, 0));
+  return KV_OK;
+}
+
 kv_status_t kvattn_set_shared_impl(int impl) {
   if (impl < 0 || impl > 2) return KV_ERR_INVALID;
   g_shared_impl.store(impl);

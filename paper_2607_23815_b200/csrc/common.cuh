@@ -77,6 +77,15 @@ struct kv_pool {
   // second stream + events used by attn_mixed to overlap the two kinds of work
   cudaStream_t side_stream;
   cudaEvent_t ev_fork, ev_join;
+  // attn_extend_host: copies in and out run on streams of their own, so that they overlap the kernels of the
+  // neighbouring steps; per staging area (up to kHostSlots in rotation) the events that order its reuse
+  static constexpr int kHostSlots = 4;
+  cudaStream_t h2d_stream, d2h_stream;
+  struct HostSlot {
+    void* staging;
+    cudaEvent_t in, ran, out;  // inputs copied in; kernels finished; results copied out
+  } host_slots[kHostSlots];
+  int host_slot_next;
 
   kvattn::PoolView view() const {
     return kvattn::PoolView{(__nv_bfloat16*)k_base, (__nv_bfloat16*)v_base, num_pages, n_kv_heads, head_dim,

@@ -180,6 +180,8 @@ static kv_status_t pool_create_impl(int num_pages, int page_size, int n_kv_heads
   p->bytes_each = (int64_t)num_pages * n_kv_heads * (int64_t)block_bytes(head_dim);
   p->d_status = nullptr; p->d_scratch_ids = nullptr; p->poison = false;
   p->side_stream = nullptr; p->ev_fork = nullptr; p->ev_join = nullptr;
+  p->h2d_stream = nullptr; p->d2h_stream = nullptr; p->host_slot_next = 0;
+  for (auto& hs : p->host_slots) hs = kv_pool::HostSlot{nullptr, nullptr, nullptr, nullptr};
   p->mark_epoch = 0; p->evicted_total = 0;
   bool ok = cudaGetDevice(&p->device) == cudaSuccess;
   if (ok && owns) {
@@ -191,7 +193,13 @@ static kv_status_t pool_create_impl(int num_pages, int page_size, int n_kv_heads
        cudaMalloc(&p->d_scratch_ids, sizeof(int) * (size_t)num_pages) == cudaSuccess &&
        cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking) == cudaSuccess &&
        cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
-       cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) == cudaSuccess;
+       cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) == cudaSuccess &&
+       cudaStreamCreateWithFlags(&p->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
+       cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
+  for (auto& hs : p->host_slots)
+    ok = ok && cudaEventCreateWithFlags(&hs.in, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&hs.ran, cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&hs.out, cudaEventDisableTiming) == cudaSuccess;
   if (!ok) {
     kv_pool_destroy(p);
     cudaGetLastError();
@@ -231,6 +239,13 @@ kv_status_t kv_pool_destroy(kv_pool_t* p) {
   if (p->side_stream) cudaStreamDestroy(p->side_stream);
   if (p->ev_fork) cudaEventDestroy(p->ev_fork);
   if (p->ev_join) cudaEventDestroy(p->ev_join);
+  if (p->h2d_stream) cudaStreamDestroy(p->h2d_stream);
+  if (p->d2h_stream) cudaStreamDestroy(p->d2h_stream);
+  for (auto& hs : p->host_slots) {
+    if (hs.in) cudaEventDestroy(hs.in);
+    if (hs.ran) cudaEventDestroy(hs.ran);
+    if (hs.out) cudaEventDestroy(hs.out);
+  }
   delete p;
   return KV_OK;
 }

@@ -61,6 +61,8 @@ _SIGNATURES = {
     "kv_gather": (_I, [_P, _P, _I, _P, _P, _P]),
     "attn_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I, _I]),
     "attn_extend": (_I, [_P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
+    "attn_extend_host_staging_bytes": (_SZ, [_P, _I, _I, _I, _I, _I]),
+    "attn_extend_host": (_I, [_P, _P, _P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_extend_shared_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I]),
     "attn_extend_shared": (_I, [_P, _P, _I, _P, _P, _P, _I, _P, _P, _I, _P, _I, _I, _I, _I, _I, _I, _F, _P, _P, _P, _SZ,
                                 _P]),
@@ -253,6 +255,26 @@ def attn_extend(pool: Pool, q, cu_q, block_tables, prefix_lens, extend_lens, max
                              _dev_ptr(out), _dev_ptr(lse), _dev_ptr(workspace),
                              0 if workspace is None else workspace.numel() * workspace.element_size(),
                              _stream(stream)), "attn_extend")
+
+
+def attn_extend_host_staging_bytes(pool: Pool, n_q_heads, batch, total_q, max_pages, max_total_len) -> int:
+    return lib().attn_extend_host_staging_bytes(pool.handle, n_q_heads, batch, total_q, max_pages, max_total_len)
+
+
+def attn_extend_host(pool: Pool, q, k_new, v_new, cu_q, block_tables, prefix_lens, extend_lens, max_extend_len,
+                     max_total_len, scale, out, lse, staging, stream=None):
+    """One step from host tensors (pinned for asynchrony): copies in, kv_append of the suffix, attn_extend, copies out.
+    `staging` is a device byte tensor of attn_extend_host_staging_bytes() bytes."""
+    for t in (q, k_new, v_new, cu_q, block_tables, prefix_lens, extend_lens, out, lse):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("attn_extend_host takes contiguous host tensors")
+    _check(lib().attn_extend_host(pool.handle, C.c_void_p(q.data_ptr()), C.c_void_p(k_new.data_ptr()),
+                                  C.c_void_p(v_new.data_ptr()), q.shape[1], C.c_void_p(cu_q.data_ptr()),
+                                  C.c_void_p(block_tables.data_ptr()), block_tables.shape[1],
+                                  C.c_void_p(prefix_lens.data_ptr()), C.c_void_p(extend_lens.data_ptr()),
+                                  prefix_lens.numel(), q.shape[0], max_extend_len, max_total_len, float(scale),
+                                  C.c_void_p(out.data_ptr()), C.c_void_p(lse.data_ptr()), _dev_ptr(staging),
+                                  staging.numel() * staging.element_size(), _stream(stream)), "attn_extend_host")
 
 
 def kvattn_set_shared_impl(impl: int):

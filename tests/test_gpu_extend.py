@@ -138,3 +138,39 @@ def test_many_one_step_items_on_the_tensor_core_kernel():
         else:
             assert np.array_equal(res["o_bits"], first)
     dp.close()
+
+
+def test_one_call_from_host_buffers_matches_append_then_extend():
+    # attn_extend_host = copies in + kv_append(suffix) + attn_extend + copies out: bit-identical to doing the
+    # same with device tensors, and within tolerance of the oracle.
+    geom = synth.Geometry(32, 8, 128)
+    P = [0, 17, 160, 500, 31]
+    E = [40, 1, 129, 64, 300]
+    dp = DualPool(geom, 128, seed=311)
+    b = Batch(dp, [p + e for p, e in zip(P, E)])
+    b.write([(i, 0, P[i]) for i in range(len(P))])                       # the upstream operator's prefix only
+    ks, vs = zip(*[b.kv(i, P[i], P[i] + E[i]) for i in range(len(P))])
+    q = torch.cat([b.q(i, P[i], P[i] + E[i]) for i in range(len(P))]).contiguous()
+    k_new, v_new = torch.cat(ks).contiguous(), torch.cat(vs).contiguous()
+    cu = torch.tensor(np.concatenate([[0], np.cumsum(E)]), dtype=torch.int32)
+    bt = torch.from_numpy(b.block_tables()).to(torch.int32).contiguous()
+    pl, el = torch.tensor(P, dtype=torch.int32), torch.tensor(E, dtype=torch.int32)
+    pin = lambda t: t.cpu().contiguous().pin_memory()
+    h = [pin(t) for t in (q, k_new, v_new, cu, bt, pl, el)]
+    out_h = torch.full(q.shape, float("nan"), dtype=torch.bfloat16).pin_memory()
+    lse_h = torch.full((q.shape[0], geom.n_q_heads), float("nan"), dtype=torch.float32).pin_memory()
+    max_l = max(p + e for p, e in zip(P, E))
+    staging = torch.empty(kvattn.attn_extend_host_staging_bytes(dp.pool, geom.n_q_heads, len(P), int(q.shape[0]),
+                                                                bt.shape[1], max_l), dtype=torch.uint8, device="cuda")
+    kvattn.attn_extend_host(dp.pool, h[0], h[1], h[2], h[3], h[4], h[5], h[6], max(E), max_l, geom.scale, out_h, lse_h,
+                            staging)
+    torch.cuda.synchronize()
+    assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+    # the oracle's pool gets the same suffix rows; the device rows were written by the call itself
+    for i in range(len(P)):
+        dp.host.append(b.rows[i], P[i], synth.bf16_bits(ks[i]), synth.bf16_bits(vs[i]))
+    res = run_extend(dp, b, P, E, impl=0)
+    assert np.array_equal(synth.bf16_bits(out_h), res["o_bits"])
+    assert np.array_equal(lse_h.numpy(), res["lse_raw"])
+    assert_close(res, "host-buffer step")
+    dp.close()
