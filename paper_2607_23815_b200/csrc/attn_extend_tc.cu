@@ -551,7 +551,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
               // tile and first K tile are already there, its first S is issued now instead of after tile 1.
               const uint32_t k0 = loads + (more ? 0 : 0) + 2 * (uint32_t)(it.ld_tiles - 1 - j) - (more ? 1 : 0);
               const uint32_t st0 = k0 % Cfg::kStages;
-              if (__all_sync(0xffffffffu, mbar_test_wait(bar_q_full, items_done[0] & 1) &&
+              // (A stage's barrier may only be asked about load k0 once the stage's previous load, k0 - kStages, has
+              // been waited for: otherwise the parity test would be answered by the phase before that one.  In the
+              // fan-out mode tile 1 can have several steps more than tile 0, which puts k0 that far ahead.)
+              if (k0 < loads + Cfg::kStages &&
+                  __all_sync(0xffffffffu, mbar_test_wait(bar_q_full, items_done[0] & 1) &&
                                               mbar_test_wait(smem_u32(&sm.kv_full[st0]), (k0 / Cfg::kStages) & 1))) {
                 ++items_done[0];
                 early0 = true;
