@@ -130,7 +130,7 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
                                                               const int* __restrict__ extend_lens,
                                                               const int* __restrict__ cu_q, int batch, int max_tp,
                                                               int lg, int max_steps, int capacity, int max_pages,
-                                                              int mode, FanArgs fan,
+                                                              int mode, FanArgs fan, int groups,
                                                               int* status, int4* __restrict__ items,
                                                               int* __restrict__ n_items, int* __restrict__ next_item,
                                                               int first_free_item) {
@@ -139,9 +139,14 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
   for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const int64_t n = (int64_t)batch * max_tp;
-  auto key_of = [&](int steps) {
-    const int64_t k = max_steps < kPlanBuckets ? steps : (int64_t)steps * (kPlanBuckets - 1) / max_steps;
-    return (int)min((int64_t)(kPlanBuckets - 1), k);
+  // Sort key, larger = earlier: the sequences are taken group after group (a group's K/V stays in L2 while its items
+  // run, and the tile pairs of a sequence read the same pages), heaviest item first inside a group.
+  const int per_group = kPlanBuckets / groups;
+  auto key_of = [&](int steps, int seq) {
+    const int64_t k = (int64_t)steps * (per_group - 1) / max(max_steps, 1);
+    const int cost = (int)min((int64_t)(per_group - 1), k);
+    const int grp = (int)((int64_t)seq * groups / batch);
+    return (groups - 1 - grp) * per_group + cost;
   };
   for (int64_t e = threadIdx.x; e < n; e += blockDim.x) {
     const int seq = (int)(e / max_tp), tp = (int)(e % max_tp);
@@ -150,7 +155,7 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
     if (((tp * 256) >> lg) >= E) continue;
     const ItemRec r = make_item(seq, tp, P, E, __ldg(cu_q + seq), lg, max_pages, mode, fan);
     const int steps = r.n_kv0 + r.n_kv1;
-    if (steps > 0) atomicAdd(&hist[key_of(steps)], 1);
+    if (steps > 0) atomicAdd(&hist[key_of(steps, seq)], 1);
   }
   __syncthreads();
   // exclusive prefix over the buckets, heaviest first: thread i owns buckets B-1-2i and B-2-2i
@@ -192,7 +197,7 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
     const int steps = r.n_kv0 + r.n_kv1;
     if (steps == 0 && (mode == 0 || P > 0 || mode == 2)) report(status, KV_ERR_BOUNDS);  // rows exist but the lengths do not fit the tables
     if (steps > 0) {
-      const int pos = atomicAdd(&hist[key_of(steps)], 1);
+      const int pos = atomicAdd(&hist[key_of(steps, seq)], 1);
       if (pos < capacity) {
         items[2 * pos] = make_int4(r.seq, r.tp, r.P, r.E);
         items[2 * pos + 1] = make_int4(r.row0, r.n_kv0, r.n_kv1, r.kv_end);
@@ -958,9 +963,16 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
     const kv_status_t gs = tc_grid(n_bound, cta_cap, &grid);
     if (gs != KV_OK) return gs;
   }
+  // about a hundred items per group (measured on the 8B extend, long-document and fan-out shapes: fewer and larger
+  // groups lose the L2 reuse, one sequence per group loses balance when a sequence has few items)
+  // (a batch with fewer than a dozen items per SM is left in pure cost order: there the balance matters more)
+  int groups = n_bound >= 12 * 148 ? n_bound / 96 : 1;
+  groups = groups < 1 ? 1 : groups;
+  groups = groups > batch ? batch : groups;
+  groups = groups > kPlanBuckets / 16 ? kPlanBuckets / 16 : groups;
   extend_tc_plan_kernel<<<1, 1024, 0, st>>>(prefix_lens, extend_lens, cu_q, batch, max_tp, lg, max_steps, (int)capacity,
-                                            max_pages, mode, fan != nullptr ? *fan : FanArgs{}, p->d_status, items, n_items,
-                                            n_items + 1, grid);
+                                            max_pages, mode, fan != nullptr ? *fan : FanArgs{}, groups, p->d_status, items,
+                                            n_items, n_items + 1, grid);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
 
