@@ -38,6 +38,8 @@ using namespace ptx;
 constexpr int kTcThreads = 512;
 constexpr int kWarpEpilogue = 8, kWarpProducer = 12, kWarpMma = 13, kWarpQ = 14;
 constexpr int kPlanBuckets = 2048;
+constexpr int kPlanSeqBuckets = 1024;   // length buckets for ranking the sequences (one per plan thread)
+constexpr int kPlanMaxRanked = 8192;    // batches up to this size are ranked by length; larger ones keep their order
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more than this
 
 struct TcArgs {
@@ -139,13 +141,63 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
   for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const int64_t n = (int64_t)batch * max_tp;
+  // The sequences are put into groups longest first, so that the last groups, which decide how evenly the CTAs
+  // finish, hold the cheapest items: a counting sort of the sequences on their length (ties in arrival order: only
+  // the order of execution depends on it).
+  __shared__ int seq_hist[kPlanSeqBuckets];
+  __shared__ unsigned short seq_rank[kPlanMaxRanked];
+  const bool ranked = groups > 1 && batch <= kPlanMaxRanked;
+  if (ranked) {
+    __shared__ int seq_warp_tot[32];
+    seq_hist[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t span = (int64_t)max(max_steps, 1) * 64 + 1;  // longer than any sequence the tables can hold
+    auto bucket_of = [&](int P, int E) {
+      return (int)min((int64_t)(kPlanSeqBuckets - 1), (int64_t)(P + E) * kPlanSeqBuckets / span);
+    };
+    for (int seq = threadIdx.x; seq < batch; seq += blockDim.x) {
+      const int P = __ldg(prefix_lens + seq), E = __ldg(extend_lens + seq);
+      if (P >= 0 && E > 0) atomicAdd(&seq_hist[bucket_of(P, E)], 1);
+    }
+    __syncthreads();
+    {  // exclusive prefix, longest bucket first: thread i owns bucket B-1-i
+      const int b = kPlanSeqBuckets - 1 - (int)threadIdx.x;
+      const int c = seq_hist[b];
+      int incl = c;
+      const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+#pragma unroll
+      for (int off = 1; off < 32; off <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, off);
+        if (lane >= off) incl += v;
+      }
+      if (lane == 31) seq_warp_tot[w] = incl;
+      __syncthreads();
+      if (w == 0) {
+        int t = seq_warp_tot[lane];
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, t, off);
+          if (lane >= off) t += v;
+        }
+        seq_warp_tot[lane] = t;
+      }
+      __syncthreads();
+      seq_hist[b] = (w > 0 ? seq_warp_tot[w - 1] : 0) + incl - c;
+    }
+    __syncthreads();
+    for (int seq = threadIdx.x; seq < batch; seq += blockDim.x) {
+      const int P = __ldg(prefix_lens + seq), E = __ldg(extend_lens + seq);
+      seq_rank[seq] = (P >= 0 && E > 0) ? (unsigned short)atomicAdd(&seq_hist[bucket_of(P, E)], 1) : 0;
+    }
+    __syncthreads();
+  }
   // Sort key, larger = earlier: the sequences are taken group after group (a group's K/V stays in L2 while its items
   // run, and the tile pairs of a sequence read the same pages), heaviest item first inside a group.
   const int per_group = kPlanBuckets / groups;
   auto key_of = [&](int steps, int seq) {
     const int64_t k = (int64_t)steps * (per_group - 1) / max(max_steps, 1);
     const int cost = (int)min((int64_t)(per_group - 1), k);
-    const int grp = (int)((int64_t)seq * groups / batch);
+    const int grp = (int)((int64_t)(ranked ? (int)seq_rank[seq] : seq) * groups / batch);
     return (groups - 1 - grp) * per_group + cost;
   };
   for (int64_t e = threadIdx.x; e < n; e += blockDim.x) {
