@@ -174,3 +174,47 @@ def test_one_call_from_host_buffers_matches_append_then_extend():
     assert np.array_equal(lse_h.numpy(), res["lse_raw"])
     assert_close(res, "host-buffer step")
     dp.close()
+
+
+class _SpikyBatch(Batch):
+    """Keys at a few chosen positions are large and aligned with every query, so that the row maximum jumps by
+    tens of binades when their tile arrives."""
+
+    def __init__(self, dp, lengths, spikes):
+        super().__init__(dp, lengths)
+        self.spikes = spikes  # {position: gain}
+        g = dp.geom
+        rng = np.random.default_rng(4242)
+        self.pattern = torch.tensor(rng.choice([-1.0, 1.0], size=g.head_dim), dtype=torch.float32, device=dp.device)
+
+    def kv(self, i, lo, hi):
+        k, v = super().kv(i, lo, hi)
+        for pos, gain in self.spikes.items():
+            if lo <= pos < hi:
+                k[pos - lo] = (gain * self.pattern).to(torch.bfloat16)
+        return k, v
+
+    def q(self, i, lo, hi):
+        return (super().q(i, lo, hi).float() + self.pattern).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("total", [2300, 4500])
+def test_scores_that_jump_far_above_the_running_maximum(total):
+    # q.k at the spikes is about gain * head_dim, i.e. tens of binades above everything seen before: the kernel
+    # variant for long sequences (total >= 4096), which assumes that the maximum in use still serves, has to notice
+    # and take such a step again with the exact maximum; the variant for short ones rescales.  Each later spike is
+    # larger than the one before, one of them sits among the suffix tokens.
+    geom = synth.Geometry(8, 2, 128)
+    _skip_if_no_tc(2, geom)
+    E = 48
+    P = total - E
+    # the last one lifts the score by more than 128 binades: without the second look its exponential is infinite
+    spikes = {700: 0.75, 1500: 1.5, total - 900: 2.5, total - 20: 9.0}
+    dp = DualPool(geom, synth.pages_needed(total, 16) + 4, seed=991)
+    b = _SpikyBatch(dp, [total], spikes)
+    b.write([(0, 0, total)])
+    for impl in (2, 1):
+        res = run_extend(dp, b, [P], [E], impl=impl)
+        assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+        assert_close(res, f"spikes, impl {impl}")
+    dp.close()
