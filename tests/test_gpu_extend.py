@@ -218,3 +218,23 @@ def test_scores_that_jump_far_above_the_running_maximum(total):
         assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
         assert_close(res, f"spikes, impl {impl}")
     dp.close()
+
+
+def test_more_sequences_than_the_plan_ranks():
+    # The plan kernel ranks the sequences of a batch by length up to a fixed batch size and keeps the batch order
+    # beyond it; groups are formed (and the ranking used) only when the batch has a dozen items per SM or more.
+    # Both sides of that size are run on the tensor-core kernel and compared with the oracle.
+    geom = synth.Geometry(8, 2, 64)
+    _skip_if_no_tc(2, geom)
+    rng = np.random.default_rng(5)
+    for n in (8300, 2200):
+        E = rng.integers(1, 5, size=n).tolist()
+        P = rng.integers(0, 40, size=n).tolist()
+        L = [p + e for p, e in zip(P, E)]
+        dp = DualPool(geom, sum(synth.pages_needed(x, 16) for x in L) + 8, seed=300 + n)
+        b = Batch(dp, L)
+        b.write([(i, 0, L[i]) for i in range(n)])
+        res = run_extend(dp, b, P, E, impl=2)
+        assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+        assert_close(res, f"{n} sequences")
+        dp.close()
