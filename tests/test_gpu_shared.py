@@ -113,3 +113,18 @@ def test_fanout_workload_shape(impl):
     child_lens = rng.integers(30, 45, size=51).tolist()
     res = _run_shared(geom, parent_lens, n_child, child_lens, seed=917, also_aliased=False, impl=impl)
     assert_close(res, f"fan-out slice impl{impl}")
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_long_parents_use_the_long_sequence_kernel(impl):
+    # parents of 4096 tokens and more select the kernel variant that does not search for the row maximum after an
+    # item's first tile; one parent is empty, so its children's rows see nothing until their own tile arrives
+    geom = synth.Geometry(16, 4, 128)
+    rng = np.random.default_rng(41)
+    parent_lens = [4400, 0, 4112]
+    n_child = [6, 3, 9]
+    child_lens = rng.integers(1, 70, size=18).tolist()
+    res = _run_shared(geom, parent_lens, n_child, child_lens, seed=941, impl=impl)
+    assert_close(res, f"long parents impl{impl}")
+    assert np.max(np.abs(res["o"] - res["o_alias"])) <= 2e-2
+    assert np.max(np.abs(res["lse"] - res["lse_alias"])) <= 1e-3
