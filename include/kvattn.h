@@ -23,6 +23,8 @@
  *    once with nothing launched.  Problems only the device can see (a block-table entry
  *    outside the pool) make the kernel skip the access and record KV_ERR_BOUNDS in a
  *    device status word that kv_last_async_status() reads.  Nothing aborts, traps or throws.
+ *  - A pool lives on the device that was current when it was created; calls that launch work must be
+ *    made with that device current (KV_ERR_INVALID otherwise).
  *  - Supported shapes: bf16 K/V/Q/O, page_size 16, head_dim 64 or 128,
  *    group G = n_q_heads / n_kv_heads in {1, 2, 4, 8}.  Anything else: KV_ERR_UNSUPPORTED.
  *  - All integer arrays are int32.  Block tables are row-major [rows][max_pages]; entry b
@@ -67,7 +69,7 @@ typedef enum {
 
 const char* kv_status_str(kv_status_t s);
 
-/* ---- pool: "a global pool of fixed-size blocks" (Section 2.1, vLLM memory model) ---------- */
+/* ---- pool: one pool of equally sized pages for all requests (Section 2.1, vLLM memory model) -- */
 
 /* Creates a pool on the current CUDA device and allocates its K and V buffers with cudaMalloc
  * (2 * num_pages * n_kv_heads * page_size * head_dim * 2 bytes).  *out receives the handle. */
@@ -92,14 +94,14 @@ kv_status_t kv_pool_set_poison(kv_pool_t* pool, int on);
 /* ---- allocator (host; mutex-guarded) ------------------------------------------------------ */
 
 /* Hands out n page ids into out_page_ids [host].  All-or-nothing: KV_ERR_OOM leaves the pool
- * unchanged ("if insufficient blocks are available, new requests are deferred", Section 2.1).
+ * unchanged; the caller holds the request back until pages are free again (Section 2.1).
  * Order is deterministic: a fresh pool gives 0,1,2,...; released pages come back last-in-first-out. */
 kv_status_t kv_alloc(kv_pool_t* pool, int n, int* out_page_ids);
 /* Returns pages whose owner is done (Algorithm 1, Complete: releaseMemory).  A page id that is out
  * of range, not allocated, or listed twice gives KV_ERR_NOT_ALLOCATED with no partial effect. */
 kv_status_t kv_free(kv_pool_t* pool, const int* page_ids /*host*/, int n);
-/* Returns pages reclaimed under memory pressure (Section 2.1: completed requests' blocks "may be
- * evicted at any time").  Same as kv_free plus the eviction counter and the optional poison fill;
+/* Returns pages reclaimed under memory pressure (Section 2.1: the blocks of a finished request stay
+ * cached only until the engine needs the room).  Same as kv_free plus the eviction counter and the optional poison fill;
  * the former owner must treat its prefix as lost and re-prefill (Section 2.2). */
 kv_status_t kv_evict(kv_pool_t* pool, const int* page_ids /*host*/, int n);
 
@@ -126,8 +128,8 @@ kv_status_t kv_evict_lru(kv_pool_t* pool, int n, int* out_page_ids /*host [n]*/,
 /* Test surface: state of one page (any pointer may be NULL). */
 kv_status_t kv_page_info(const kv_pool_t* pool, int page, int* allocated, int* refs, int* pins);
 
-/* ---- kv_append: materialise new tokens' K/V in their pages (Section 2.1: prefill "materializes
- *      per-layer key-value tensors") ------------------------------------------------------- */
+/* ---- kv_append: store new tokens' K/V in their pages (Section 2.1: prefill produces the K/V
+ *      tensors of every prompt token, layer by layer) ---------------------------------------- */
 /* n_segments segments; segment s holds rows cu_new[s] .. cu_new[s+1]-1 of k_new/v_new
  * ([dev] bf16 [total_new][n_kv_heads][head_dim]) and writes them to token positions
  * start_pos[s] .. of the sequence whose block-table row is seg_row[s] (seg_row NULL: row s).
@@ -156,13 +158,15 @@ kv_status_t kv_gather(kv_pool_t* pool, const int* block_table_row, int len, void
 size_t attn_workspace_bytes(const kv_pool_t* pool, int n_q_heads, int batch_ext, int total_q, int max_total_len,
                             int batch_dec, int max_ctx_len);
 
-/* Extend ("only prefills the ... suffix", Section 2.1): sequence i has prefix_lens[i] reused tokens
+/* Extend (the downstream operator prefills nothing but its own suffix, Section 2.1): sequence i has prefix_lens[i] reused tokens
  * and extend_lens[i] new ones, all already in its pages (kv_append first).  Suffix token t sits at
  * position prefix_lens[i]+t and sees keys 0..prefix_lens[i]+t.  prefix_lens[i]=0 is a from-scratch
  * prefill (the cache-miss path of Section 2.2); extend_lens[i]=0 contributes no rows.
  * q/out [dev] bf16 [total_q][n_q_heads][head_dim], ragged by cu_q [dev][batch+1]; lse [dev] fp32
  * [total_q][n_q_heads]; prefix_lens, extend_lens [dev][batch].  max_extend_len / max_total_len are
- * host-side upper bounds on extend_lens[i] and prefix_lens[i]+extend_lens[i] (they size the grid). */
+ * host-side upper bounds on extend_lens[i] and prefix_lens[i]+extend_lens[i] (they size the grid); a
+ * sequence that exceeds them on the device, or suffix rows beyond total_q, is recorded as KV_ERR_BOUNDS
+ * (kv_last_async_status) and its rows beyond the bound are left unwritten. */
 kv_status_t attn_extend(kv_pool_t* pool, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                         int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                         int max_extend_len, int max_total_len, float scale, void* out, float* lse,
@@ -218,7 +222,7 @@ kv_status_t attn_extend_shared(kv_pool_t* pool, const void* q, int n_q_heads, co
                                int max_parent_len, float scale, void* out, float* lse, void* workspace,
                                size_t workspace_bytes, void* stream);
 
-/* Decode ("one token at a time, attending over all previously computed KV", Section 2.1): one query
+/* Decode (each new token attends over every K/V stored so far, Section 2.1): one query
  * per sequence at position ctx_lens[i]-1 over keys 0..ctx_lens[i]-1 (its own K/V already appended).
  * q/out [dev] bf16 [batch][n_q_heads][head_dim]; lse [dev] fp32 [batch][n_q_heads]; ctx_lens [dev]
  * [batch]; max_ctx_len: host upper bound.  ctx_lens[i] <= 0 writes O = 0, LSE = -inf. */
@@ -260,7 +264,9 @@ typedef struct {
  * extend set and the decode set are launched so that the tensor-bound and the HBM-bound work
  * share the GPU.  Either argument may be NULL or have batch 0.  The workspace must be sized by
  * attn_workspace_bytes() with both batches.  Work is ordered after prior work on `stream`, and
- * later work on `stream` is ordered after it. */
+ * later work on `stream` is ordered after it.  The call uses a side stream and a pair of events that
+ * belong to the pool: two attn_mixed calls on the same pool must not be issued concurrently from two
+ * threads, nor on two different caller streams without an ordering between them. */
 kv_status_t attn_mixed(kv_pool_t* pool, int n_q_heads, float scale, const attn_extend_args_t* ext,
                        const attn_decode_args_t* dec, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -282,6 +288,13 @@ kv_status_t kvattn_set_shared_impl(int impl);
 /* Tuning: inside attn_mixed (both sets present) the persistent extend kernel takes at most n SMs, so that the
  * HBM-bound decode kernel runs beside it on the others instead of after it.  0 = no limit.  Process-wide. */
 kv_status_t kvattn_set_mixed_extend_ctas(int n);
+/* Test surface (the paper has no counterpart): runs a one-CTA kernel whose warps wait, with the same bounded
+ * wait the attention kernels use, on barriers that nothing completes; the first gives up after limit_ns
+ * (1 .. 1e8), raises the CTA's abort flag, which releases the others, the kernel frees its tensor memory and
+ * records KV_ERR_TIMEOUT, which kv_last_async_status() then returns (and clears).  The device stays usable.
+ * trace [dev][4] receives: bulk copy landed (1), lanes that gave up (32), parked warp released by the flag (1),
+ * nanoseconds waited. */
+kv_status_t kvattn_selftest_bounded_wait(kv_pool_t* pool, unsigned long long limit_ns, int* trace, void* stream);
 /* Number of kernels this library has launched since load (all pools); for benchmark accounting. */
 int64_t kvattn_launch_count(void);
 

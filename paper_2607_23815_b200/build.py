@@ -13,7 +13,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvattn.so")
-SOURCES = ["pool.cu", "attn_small.cu", "attn_extend_tc.cu", "attn_decode_static.cu", "attn_shared.cu", "api.cu"]
+SOURCES = ["pool.cu", "attn_small.cu", "attn_extend_tc.cu", "attn_decode_static.cu", "attn_shared.cu", "selftest.cu", "api.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "--shared", "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

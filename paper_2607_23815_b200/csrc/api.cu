@@ -72,6 +72,7 @@ static kv_status_t extend_impl(kv_pool_t* p, const void* q, int n_q_heads, const
     return KV_ERR_INVALID;
   if ((((uintptr_t)q) | ((uintptr_t)out)) & 15) return KV_ERR_INVALID;
   if (max_total_len < max_extend_len || max_total_len > (int64_t)max_pages * kPageSize) return KV_ERR_INVALID;
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
   const int impl = g_extend_impl.load();
   const bool tc_ok = extend_tc_supported(p, n_q_heads) && scale > 0.f;  // the tensor-core kernel folds a positive scale into the row maximum
   if (impl == 2 && !tc_ok) return KV_ERR_UNSUPPORTED;
@@ -117,6 +118,7 @@ kv_status_t attn_extend_shared(kv_pool_t* p, const void* q, int n_q_heads, const
       max_parent_rows < max_child_len)
     return KV_ERR_INVALID;
   if (!(scale > 0.f) || !extend_tc_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
   return launch_extend_shared(p, q, n_q_heads, cu_q, cu_children, parent_tables, max_pages_parent, parent_lens, child_tables,
                               max_pages_child, child_lens, n_parents, n_children, total_q, max_child_len, max_parent_rows,
                               max_parent_len, scale, out, lse, workspace, workspace_bytes, (cudaStream_t)stream);
@@ -166,6 +168,7 @@ kv_status_t attn_extend_host(kv_pool_t* p, const void* q, const void* k_new, con
       prefix_lens == nullptr || extend_lens == nullptr || out == nullptr || lse == nullptr || staging == nullptr)
     return KV_ERR_INVALID;
   if (((uintptr_t)staging) & 255) return KV_ERR_INVALID;
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
   const HostStepLayout L = host_step_layout(p, n_q_heads, batch, total_q, max_pages, max_total_len);
   if (staging_bytes < L.total) return KV_ERR_WORKSPACE;
   cudaStream_t st = (cudaStream_t)stream;
@@ -241,6 +244,7 @@ kv_status_t attn_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* b
     return KV_ERR_INVALID;
   if ((((uintptr_t)q) | ((uintptr_t)out)) & 15) return KV_ERR_INVALID;
   if (max_ctx_len > (int64_t)max_pages * kPageSize) return KV_ERR_INVALID;
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
   if (max_ctx_len == 0) max_ctx_len = 1;  // every row is empty: still defines O = 0, LSE = -inf
   // the decode region of a combined workspace starts after the extend region; a caller that sized
   // the workspace for decode only passes (0, 0) for the extend part, so the offset is 0 there
@@ -250,7 +254,7 @@ kv_status_t attn_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* b
 
 kv_status_t attn_mixed(kv_pool_t* p, int n_q_heads, float scale, const attn_extend_args_t* ext,
                        const attn_decode_args_t* dec, void* workspace, size_t workspace_bytes, void* stream) {
-  if (p == nullptr) return KV_ERR_INVALID;
+  if (p == nullptr || !on_pool_device(p)) return KV_ERR_INVALID;
   if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
   const bool has_ext = ext != nullptr && ext->batch > 0 && ext->total_q > 0;
   const bool has_dec = dec != nullptr && dec->batch > 0;

@@ -20,7 +20,6 @@ constexpr size_t kStaticScratchBytes = size_t(8) << 20;  // 8 MiB, held by every
 // combine step reads only the slots that the same call wrote before.
 static __device__ __align__(256) unsigned char g_decode_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
 static std::mutex g_scratch_mu;
 static void* g_scratch_ptr[kMaxDevices] = {};  // device address of g_decode_scratch, per device
 
@@ -57,6 +56,8 @@ extern "C" kv_status_t attn_decode_static(kv_pool_t* p, const void* q, int n_q_h
     return KV_ERR_INVALID;
   if ((((uintptr_t)q) | ((uintptr_t)out)) & 15) return KV_ERR_INVALID;
   if (max_ctx_len > (int64_t)max_pages * kPageSize) return KV_ERR_INVALID;
+  // the array's address is taken for the current device: that has to be the device that holds the pool's pages
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
   if (max_ctx_len == 0) max_ctx_len = 1;
   // the batch must fit the fixed scratch: refuse, do not truncate
   const size_t need = decode_workspace_bytes(n_q_heads, p->head_dim, batch, max_ctx_len);

@@ -143,6 +143,12 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
   for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
   __syncthreads();
   const int64_t n = (int64_t)batch * max_tp;
+  // A sequence with more suffix tokens than the host-side bound the grid was sized with would lose its last rows
+  // without a trace: it is reported instead.
+  for (int seq = threadIdx.x; seq < batch; seq += blockDim.x) {
+    const int E = __ldg(extend_lens + seq);
+    if (__ldg(prefix_lens + seq) >= 0 && (int64_t)E > (((int64_t)max_tp * 256) >> lg)) report(status, KV_ERR_BOUNDS);
+  }
   // The sequences are put into groups longest first, so that the last groups, which decide how evenly the CTAs
   // finish, hold the cheapest items: a counting sort of the sequences on their length (ties in arrival order: only
   // the order of execution depends on it).
@@ -255,6 +261,8 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
       if (pos < capacity) {
         items[2 * pos] = make_int4(r.seq, r.tp, r.P, r.E);
         items[2 * pos + 1] = make_int4(r.row0, r.n_kv0, r.n_kv1, r.kv_end);
+      } else {
+        report(status, KV_ERR_BOUNDS);  // more rows on the device than the total the host gave: the entry is dropped
       }
     }
   }
@@ -1029,13 +1037,8 @@ static kv_status_t make_q_map(CUtensorMap* map, const void* q, int total_q, int 
 }
 
 // One persistent CTA per SM, fewer if there are fewer items or the caller caps the kernel.
-static kv_status_t tc_grid(int n_items_bound, int cta_cap, int* grid_out) {
-  static int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    KV_CUDA_OK(cudaGetDevice(&dev));
-    KV_CUDA_OK(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
-  }
+static kv_status_t tc_grid(const kv_pool_t* p, int n_items_bound, int cta_cap, int* grid_out) {
+  const int sm_count = sm_count_of(p->device);
   int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
   if (cta_cap > 0 && grid > cta_cap) grid = cta_cap;  // leave the other SMs to work that runs beside this kernel
   *grid_out = grid;
@@ -1043,12 +1046,13 @@ static kv_status_t tc_grid(int n_items_bound, int cta_cap, int* grid_out) {
 }
 
 template <int D, bool OPT>
-static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid, cudaStream_t st) {
+static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid, int device, cudaStream_t st) {
   const size_t smem = sizeof(TcSmem<D>);
-  static bool configured = false;
-  if (!configured) {
+  static std::atomic<bool> configured[kMaxDevices];  // the attribute belongs to the function on one device
+  if (device < 0 || device >= kMaxDevices) return KV_ERR_INVALID;
+  if (!configured[device].load(std::memory_order_acquire)) {
     KV_CUDA_OK(cudaFuncSetAttribute(attn_extend_tc_kernel<D, OPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    configured = true;
+    configured[device].store(true, std::memory_order_release);
   }
   attn_extend_tc_kernel<D, OPT><<<grid, kTcThreads, smem, st>>>(a, q_map);
   count_launch();
@@ -1082,13 +1086,13 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   const int n_bound = bound > (1 << 30) ? (1 << 30) : (int)bound;
   int grid = 1;
   {
-    const kv_status_t gs = tc_grid(n_bound, cta_cap, &grid);
+    const kv_status_t gs = tc_grid(p, n_bound, cta_cap, &grid);
     if (gs != KV_OK) return gs;
   }
   // about a hundred items per group (measured on the 8B extend, long-document and fan-out shapes: fewer and larger
   // groups lose the L2 reuse, one sequence per group loses balance when a sequence has few items)
   // (a batch with fewer than a dozen items per SM is left in pure cost order: there the balance matters more)
-  int groups = n_bound >= 12 * 148 ? n_bound / 96 : 1;
+  int groups = n_bound >= 12 * sm_count_of(p->device) ? n_bound / 96 : 1;
   groups = groups < 1 ? 1 : groups;
   groups = groups > batch ? batch : groups;
   groups = groups > kPlanBuckets / 16 ? kPlanBuckets / 16 : groups;
@@ -1121,8 +1125,9 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   // Skipping the search for the row maximum pays where items have many KV steps (measured: +2 % on the
   // long-document shapes, -1 % on the 8B extend batch whose items have a dozen steps)
   const bool opt = max_total_len >= kOptimisticMinLen;
-  if (p->head_dim == 128) return opt ? launch_tc<128, true>(a, q_map, grid, st) : launch_tc<128, false>(a, q_map, grid, st);
-  return opt ? launch_tc<64, true>(a, q_map, grid, st) : launch_tc<64, false>(a, q_map, grid, st);
+  if (p->head_dim == 128)
+    return opt ? launch_tc<128, true>(a, q_map, grid, p->device, st) : launch_tc<128, false>(a, q_map, grid, p->device, st);
+  return opt ? launch_tc<64, true>(a, q_map, grid, p->device, st) : launch_tc<64, false>(a, q_map, grid, p->device, st);
 }
 
 }  // namespace kvattn

@@ -139,6 +139,8 @@ __global__ void __launch_bounds__(256, 1) attn_small_kernel(SmallArgs a, int64_t
     row0 = seq;
   }
   const int tpt = EXTEND ? 8 / G : 1;  // query tokens per tile
+  // more suffix tokens than the host-side bound the grid covers: the rows beyond it would never be written
+  if (EXTEND && rt == 0 && lane == 0 && (int64_t)E > (int64_t)a.max_row_tiles * tpt) report(a.pool.status, KV_ERR_BOUNDS);
   const int t_first = rt * tpt;
   if (t_first >= E || L <= 0 || P < 0) return;
   if (L > a.max_pages * kPageSize) { report(a.pool.status, KV_ERR_BOUNDS); return; }

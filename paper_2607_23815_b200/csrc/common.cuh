@@ -51,6 +51,10 @@ struct FanArgs {
 extern std::atomic<int64_t> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+constexpr int kMaxDevices = 64;
+// Multiprocessors of the given device (asked once per device).
+int sm_count_of(int device);
+
 }  // namespace kvattn
 
 struct kv_pool {
@@ -92,6 +96,13 @@ struct kv_pool {
                             d_status};
   }
 };
+
+// A pool's kernels are launched on the calling thread's current device and must therefore find the pool's memory
+// there: launchers return KV_ERR_INVALID when the current device is not the one the pool was created on.
+inline bool on_pool_device(const kv_pool* p) {
+  int dev = -1;
+  return cudaGetDevice(&dev) == cudaSuccess && dev == p->device;
+}
 
 #define KV_CUDA_OK(expr)                      \
   do {                                        \

@@ -9,10 +9,9 @@ namespace kvattn {
 std::atomic<int64_t> g_launches{0};
 
 // ------------------------------------------------------------------------------------------
-// kv_append: one thread moves one 16-byte chunk of K and the matching chunk of V.
-// Consecutive threads read consecutive chunks of a token row (coalesced 16-byte loads); the
-// eight chunks of a 64-dim half land, permuted, in one 128-byte row of the page (full-line
-// 16-byte stores).
+// kv_append: one warp moves one token.  Its lanes read consecutive 16-byte chunks of the token's K and V
+// rows (coalesced loads, all in flight before the first store); the eight chunks of a 64-dim half land,
+// permuted, in one 128-byte row of the page (full-line 16-byte stores).
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) append_kernel(PoolView pool, const uint4* __restrict__ k_new,
                                                      const uint4* __restrict__ v_new,
@@ -137,9 +136,23 @@ static bool shape_supported(int page_size, int n_kv_heads, int head_dim) {
   return page_size == kPageSize && (head_dim == 64 || head_dim == 128) && n_kv_heads >= 1;
 }
 
-static int grid_for(int64_t work_items, int threads) {
+int sm_count_of(int device) {
+  static std::atomic<int> cached[kMaxDevices];
+  if (device < 0 || device >= kMaxDevices) return 1;
+  int n = cached[device].load(std::memory_order_relaxed);
+  if (n == 0) {
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      return 1;
+    }
+    cached[device].store(n, std::memory_order_relaxed);
+  }
+  return n;
+}
+
+static int grid_for(const kv_pool_t* p, int64_t work_items, int threads) {
   int64_t blocks = (work_items + threads - 1) / threads;
-  const int64_t cap = 148 * 16;  // a few waves of resident blocks; grid-stride covers the rest
+  const int64_t cap = (int64_t)sm_count_of(p->device) * 16;  // a few waves of resident blocks; grid-stride covers the rest
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   return (int)blocks;
@@ -439,7 +452,8 @@ kv_status_t kv_append(kv_pool_t* p, const void* k_new, const void* v_new, const 
   if (k_new == nullptr || v_new == nullptr || cu_new == nullptr || start_pos == nullptr || block_tables == nullptr)
     return KV_ERR_INVALID;
   if ((((uintptr_t)k_new) | ((uintptr_t)v_new)) & 15) return KV_ERR_INVALID;
-  append_kernel<<<grid_for((int64_t)total_new * 32, 256), 256, 0, (cudaStream_t)stream>>>(  // one warp per token
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
+  append_kernel<<<grid_for(p, (int64_t)total_new * 32, 256), 256, 0, (cudaStream_t)stream>>>(  // one warp per token
       p->view(), (const uint4*)k_new, (const uint4*)v_new, cu_new, start_pos, seg_row, block_tables, max_pages,
       n_segments, total_new);
   count_launch();
@@ -452,8 +466,9 @@ kv_status_t kv_gather(kv_pool_t* p, const int* block_table_row, int len, void* k
   if (len == 0) return KV_OK;
   if (block_table_row == nullptr || k_out == nullptr || v_out == nullptr) return KV_ERR_INVALID;
   if ((((uintptr_t)k_out) | ((uintptr_t)v_out)) & 15) return KV_ERR_INVALID;
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
   const int64_t chunks = (int64_t)len * p->n_kv_heads * (p->head_dim >> 3);
-  gather_kernel<<<grid_for(chunks, 256), 256, 0, (cudaStream_t)stream>>>(p->view(), block_table_row, len,
+  gather_kernel<<<grid_for(p, chunks, 256), 256, 0, (cudaStream_t)stream>>>(p->view(), block_table_row, len,
                                                                          (uint4*)k_out, (uint4*)v_out);
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
@@ -461,7 +476,7 @@ kv_status_t kv_gather(kv_pool_t* p, const int* block_table_row, int len, void* k
 }
 
 kv_status_t kv_last_async_status(kv_pool_t* p) {
-  if (p == nullptr) return KV_ERR_INVALID;
+  if (p == nullptr || !on_pool_device(p)) return KV_ERR_INVALID;
   int code = 0;
   KV_CUDA_OK(cudaDeviceSynchronize());
   KV_CUDA_OK(cudaMemcpy(&code, p->d_status, sizeof(int), cudaMemcpyDeviceToHost));
@@ -474,6 +489,7 @@ kv_status_t kv_check_batch(kv_pool_t* p, const int* block_tables, int max_pages,
   if (p == nullptr || batch < 0 || max_pages < 0) return KV_ERR_INVALID;
   if (batch == 0) return KV_OK;
   if (block_tables == nullptr || lens == nullptr) return KV_ERR_INVALID;
+  if (!on_pool_device(p)) return KV_ERR_INVALID;
   check_batch_kernel<<<batch < 1184 ? batch : 1184, 128, 0, (cudaStream_t)stream>>>(p->view(), block_tables,
                                                                                   max_pages, lens, batch);
   count_launch();

@@ -75,6 +75,7 @@ _SIGNATURES = {
     "kvattn_set_extend_impl": (_I, [_I]),
     "kvattn_set_shared_impl": (_I, [_I]),
     "kvattn_set_mixed_extend_ctas": (_I, [_I]),
+    "kvattn_selftest_bounded_wait": (_I, [_P, C.c_ulonglong, _P, _P]),
     "kvattn_launch_count": (_I64, []),
 }
 
@@ -353,6 +354,12 @@ def kvattn_set_extend_impl(impl: int):
 
 def kvattn_set_mixed_extend_ctas(n: int):
     _check(lib().kvattn_set_mixed_extend_ctas(n), "kvattn_set_mixed_extend_ctas")
+
+
+def kvattn_selftest_bounded_wait(pool: Pool, limit_ns: int, trace, stream=None):
+    """Test surface: lets a bounded device-side wait run out (see the header); trace is an int32 device tensor [4]."""
+    _check(lib().kvattn_selftest_bounded_wait(pool.handle, int(limit_ns), _dev_ptr(trace), _stream(stream)),
+           "kvattn_selftest_bounded_wait")
 
 
 def kvattn_launch_count() -> int:

@@ -286,3 +286,186 @@ class FanoutWorkload:
         self.pool.destroy()
         if status != kvattn.KV_OK:
             raise kvattn.KvError(status, "device status at close")
+
+
+class PipelineLoop:
+    """The two-operator pipeline step (sem_map feeding sem_filter, Section 1) as a loop over several steps at full
+    size: a decode set whose contexts grow by one token per step, an extend set that is redrawn every step, one
+    kv_append of each step's new tokens (the extend suffixes and one token per decode sequence), attn_mixed, and
+    between steps a seeded fraction of the live pages evicted, re-allocated and re-filled (an evicted block's owner
+    recomputes it, Section 2.2).  Plays the engine around the library; holds no attention arithmetic.
+
+    The K/V "source" tensors stand for what the model would recompute: values are keyed on (sequence uid, position),
+    so a re-append after an eviction writes the same bits again.
+    """
+
+    def __init__(self, w: synth.Workload, device="cuda", seed_offset: int = 0, steps: int = 8, poison: bool = False):
+        self.w, self.geom, self.device, self.steps = w, w.geom, device, steps
+        self.seed = ranks.replica_seed(w.seed, seed_offset)
+        g = w.geom
+        self.pool = kvattn.kv_pool_create(w.num_pages, g.page_size, g.n_kv_heads, g.head_dim)
+        if poison:
+            kvattn.kv_pool_set_poison(self.pool, True)
+        # random physical placement: take every page and give them back in a seeded order, so that the library's
+        # last-in-first-out free list hands them out in that order
+        ids = kvattn.kv_alloc(self.pool, w.num_pages)
+        perm = synth.page_permutation(self.seed, w.num_pages)
+        kvattn.kv_free(self.pool, [ids[i] for i in perm.tolist()])
+        _, dec = synth.draw_lengths(dataclasses.replace(w, seed=self.seed))
+        self.n_ext, self.n_dec = w.n_extend, len(dec)
+        self.ctx = list(dec)                                                   # current decode context lengths
+        self.max_pages = synth.pages_needed(max(max(dec) + steps, w.prefix_range[1] + w.extend_range[1]), g.page_size)
+        self.rows = [[] for _ in range(self.n_ext)] + \
+                    [kvattn.kv_alloc(self.pool, synth.pages_needed(c + steps, g.page_size)) for c in dec]
+        self.dec_uids = [1_000_000 + i for i in range(self.n_dec)]
+        self.dec_src_off = np.concatenate([[0], np.cumsum([c + steps for c in dec])]).astype(np.int64)
+        self.dec_k_src = torch.cat([synth.normal_bf16(self.seed, synth.TAG_K, u, 0, c + steps, g.n_kv_heads, g.head_dim, device)
+                                    for u, c in zip(self.dec_uids, dec)])
+        self.dec_v_src = torch.cat([synth.normal_bf16(self.seed, synth.TAG_V, u, 0, c + steps, g.n_kv_heads, g.head_dim, device)
+                                    for u, c in zip(self.dec_uids, dec)])
+        self.bt_host = np.full((self.n_ext + self.n_dec, self.max_pages), -1, dtype=np.int32)
+        for j in range(self.n_dec):
+            r = self.rows[self.n_ext + j]
+            self.bt_host[self.n_ext + j, :len(r)] = r
+        self.bt = torch.from_numpy(self.bt_host).to(device)
+        # the decode sequences' contexts so far (an earlier operator's work, not part of a step)
+        self._append_ranges([(self.n_ext + j, 0, dec[j]) for j in range(self.n_dec)])
+        self.step_index = -1
+        self.prefix, self.extend = [], []
+        nb = kvattn.attn_workspace_bytes(self.pool, g.n_q_heads, self.n_ext, self.n_ext * w.extend_range[1],
+                                         w.prefix_range[1] + w.extend_range[1], self.n_dec, max(dec) + steps)
+        self.workspace = torch.empty(max(nb, 256), dtype=torch.uint8, device=device)
+        torch.cuda.synchronize()
+
+    def _i32(self, x):
+        return torch.tensor(np.asarray(x), dtype=torch.int32, device=self.device)
+
+    # -- where a row's K/V come from ---------------------------------------------------------------
+    def _src(self, row):
+        """(k_src, v_src, offset of the row's token 0, tokens held)"""
+        if row < self.n_ext:
+            return self.ext_k_src, self.ext_v_src, int(self.ext_src_off[row]), self.prefix[row] + self.extend[row]
+        j = row - self.n_ext
+        return self.dec_k_src, self.dec_v_src, int(self.dec_src_off[j]), self.ctx[j]
+
+    def _append_ranges(self, ranges, slab_tokens=1 << 17):
+        """kv_append of (row, lo, hi) token ranges, rows gathered from the source tensors (extend rows and decode rows
+        in separate calls, in slabs that bound the temporary memory)."""
+        for is_ext in (True, False):
+            part = [(r, lo, hi) for r, lo, hi in ranges if (r < self.n_ext) == is_ext and hi > lo]
+            while part:
+                take, tok = [], 0
+                while part and tok < slab_tokens:
+                    take.append(part.pop()); tok += take[-1][2] - take[-1][1]
+                k_src, v_src = (self.ext_k_src, self.ext_v_src) if is_ext else (self.dec_k_src, self.dec_v_src)
+                idx = np.concatenate([np.arange(self._src(r)[2] + lo, self._src(r)[2] + hi) for r, lo, hi in take])
+                idx_d = torch.from_numpy(idx).to(self.device)
+                cu = np.concatenate([[0], np.cumsum([hi - lo for _, lo, hi in take])])
+                kvattn.kv_append(self.pool, k_src.index_select(0, idx_d), v_src.index_select(0, idx_d), self._i32(cu),
+                                 self._i32([lo for _, lo, _ in take]), self._i32([r for r, _, _ in take]), self.bt)
+                torch.cuda.synchronize()
+
+    # -- one step -----------------------------------------------------------------------------------
+    def begin_step(self):
+        """Draws this step's extend set, places it, writes the upstream operator's prefixes (not part of the step) and
+        stages the step's new tokens: the extend suffixes followed by one token per decode sequence."""
+        self.step_index += 1
+        s, w, g, dev = self.step_index, self.w, self.geom, self.device
+        n = self.n_ext
+        self.prefix = [synth.uniform_int(self.seed, synth.TAG_LEN_A, 10_000 * (s + 1) + i, *w.prefix_range) for i in range(n)]
+        self.extend = [synth.uniform_int(self.seed, synth.TAG_LEN_B, 10_000 * (s + 1) + i, *w.extend_range) for i in range(n)]
+        self.ext_uids = [10_000 * (s + 1) + i for i in range(n)]
+        L = [p + e for p, e in zip(self.prefix, self.extend)]
+        self.ext_src_off = np.concatenate([[0], np.cumsum(L)]).astype(np.int64)
+        self.ext_k_src = torch.cat([synth.normal_bf16(self.seed, synth.TAG_K, u, 0, l, g.n_kv_heads, g.head_dim, dev)
+                                    for u, l in zip(self.ext_uids, L)])
+        self.ext_v_src = torch.cat([synth.normal_bf16(self.seed, synth.TAG_V, u, 0, l, g.n_kv_heads, g.head_dim, dev)
+                                    for u, l in zip(self.ext_uids, L)])
+        for i in range(n):
+            self.rows[i] = kvattn.kv_alloc(self.pool, synth.pages_needed(L[i], g.page_size))
+            self.bt_host[i] = -1
+            self.bt_host[i, :len(self.rows[i])] = self.rows[i]
+        self.bt.copy_(torch.from_numpy(self.bt_host))
+        self._append_ranges([(i, 0, self.prefix[i]) for i in range(n)])
+        # the step's inputs
+        self.q_ext = torch.cat([synth.normal_bf16(self.seed, synth.TAG_Q, self.ext_uids[i], self.prefix[i], self.extend[i],
+                                                  g.n_q_heads, g.head_dim, dev) for i in range(n)])
+        self.q_dec = torch.cat([synth.normal_bf16(self.seed, synth.TAG_Q, self.dec_uids[j], self.ctx[j], 1, g.n_q_heads,
+                                                  g.head_dim, dev) for j in range(self.n_dec)])
+        new_idx_e = np.concatenate([np.arange(self.ext_src_off[i] + self.prefix[i], self.ext_src_off[i + 1]) for i in range(n)])
+        new_idx_d = np.asarray([self.dec_src_off[j] + self.ctx[j] for j in range(self.n_dec)])
+        self.k_new = torch.cat([self.ext_k_src.index_select(0, torch.from_numpy(new_idx_e).to(dev)),
+                                self.dec_k_src.index_select(0, torch.from_numpy(new_idx_d).to(dev))])
+        self.v_new = torch.cat([self.ext_v_src.index_select(0, torch.from_numpy(new_idx_e).to(dev)),
+                                self.dec_v_src.index_select(0, torch.from_numpy(new_idx_d).to(dev))])
+        self.cu_new = self._i32(np.concatenate([[0], np.cumsum(self.extend + [1] * self.n_dec)]))
+        self.start_new = self._i32(self.prefix + self.ctx)
+        self.cu_q = self._i32(np.concatenate([[0], np.cumsum(self.extend)]))
+        self.prefix_d, self.extend_d = self._i32(self.prefix), self._i32(self.extend)
+        self.ctx_after = [c + 1 for c in self.ctx]
+        self.ctx_d = self._i32(self.ctx_after)
+        self.out_ext, self.out_dec = torch.empty_like(self.q_ext), torch.empty_like(self.q_dec)
+        self.lse_ext = torch.empty((self.q_ext.shape[0], g.n_q_heads), dtype=torch.float32, device=dev)
+        self.lse_dec = torch.empty((self.n_dec, g.n_q_heads), dtype=torch.float32, device=dev)
+        torch.cuda.synchronize()
+
+    def append_new(self, stream=None):
+        """kv_append of the step's new tokens (sum of the extend lengths + one per decode sequence), one call."""
+        kvattn.kv_append(self.pool, self.k_new, self.v_new, self.cu_new, self.start_new, None, self.bt, stream)
+
+    def mixed(self, stream=None):
+        g, n = self.geom, self.n_ext
+        ea = kvattn.extend_args(self.q_ext, self.cu_q, self.bt[:n], self.prefix_d, self.extend_d, max(self.extend),
+                                max(p + e for p, e in zip(self.prefix, self.extend)), self.out_ext, self.lse_ext)
+        da = kvattn.decode_args(self.q_dec, self.bt[n:], self.ctx_d, max(self.ctx_after), self.out_dec, self.lse_dec)
+        kvattn.attn_mixed(self.pool, g.n_q_heads, g.scale, ea, da, self.workspace, stream)
+
+    def commit_new(self):
+        """The decode sequences now hold one token more."""
+        self.ctx = list(self.ctx_after)
+
+    def live_blocks(self):
+        """(row, logical block) of every page that holds tokens (call after commit_new)."""
+        out = []
+        for r in range(self.n_ext + self.n_dec):
+            out += [(r, b) for b in range(synth.pages_needed(self._src(r)[3], self.geom.page_size))]
+        return out
+
+    def churn(self, fraction=0.2):
+        """Evicts a seeded fraction of the live pages, takes as many new ones, and re-fills those logical blocks.
+        Returns the number of pages that moved."""
+        live = self.live_blocks()
+        rng = np.random.default_rng(self.seed % (1 << 31) + self.step_index)
+        pick = rng.choice(len(live), size=int(len(live) * fraction), replace=False)
+        victims = [live[k] for k in pick]
+        old = [self.rows[r][b] for r, b in victims]
+        kvattn.kv_evict(self.pool, old)
+        new = kvattn.kv_alloc(self.pool, len(old))                       # last-in-first-out: the same ids, another order
+        new = [new[k] for k in rng.permutation(len(new))]
+        for (r, b), pg in zip(victims, new):
+            self.rows[r][b] = pg
+            self.bt_host[r, b] = pg
+        self.bt.copy_(torch.from_numpy(self.bt_host))
+        self._append_ranges([(r, 16 * b, min(16 * b + 16, self._src(r)[3])) for r, b in victims])
+        return len(old)
+
+    def end_step(self):
+        """The extend set's tuples leave the pipeline: their pages are released (Algorithm 1, Complete)."""
+        for i in range(self.n_ext):
+            kvattn.kv_free(self.pool, self.rows[i])
+            self.rows[i] = []
+
+    def source_bits(self, row):
+        """K/V bit patterns of a row's tokens from the source tensors (the oracle's input)."""
+        k_src, v_src, off, n = self._src(row)
+        return synth.bf16_bits(k_src[off:off + n]), synth.bf16_bits(v_src[off:off + n])
+
+    def step_new_tokens(self) -> int:
+        return int(sum(self.extend)) + self.n_dec
+
+    def close(self):
+        torch.cuda.synchronize()
+        status = kvattn.kv_last_async_status(self.pool)
+        self.pool.destroy()
+        if status != kvattn.KV_OK:
+            raise kvattn.KvError(status, "device status at close")

@@ -7,7 +7,7 @@ import torch
 
 from oracle import paged_attention as orc
 from paper_2607_23815_b200 import kvattn, synth
-from paper_2607_23815_b200.workload import DeviceWorkload
+from paper_2607_23815_b200.workload import DeviceWorkload, PipelineLoop
 from harness import O_TOL, LSE_TOL, tight_ok
 
 pytestmark = pytest.mark.gpu
@@ -139,3 +139,127 @@ def test_long_document_reuse_vs_from_scratch():
     assert d_o <= O_TOL and d_l <= LSE_TOL, (d_o, d_l)
     assert kvattn.kv_last_async_status(wl.pool) == kvattn.KV_OK
     wl.close()
+
+
+def _row_sample(P, E, seed, fraction=0.25):
+    """A seeded quarter of a tuple's suffix rows that always holds the first and last row and every row whose
+    absolute position starts or ends a page."""
+    pos = P + np.arange(E)
+    must = {0, E - 1} | {int(t) for t in np.nonzero((pos % 16 == 0) | (pos % 16 == 15))[0]}
+    rng = np.random.default_rng(seed)
+    rest = np.array(sorted(set(range(E)) - must), dtype=np.int64)
+    n_extra = min(len(rest), max(0, int(np.ceil(fraction * E)) - len(must)))
+    extra = rng.choice(rest, size=n_extra, replace=False) if n_extra else []
+    return np.array(sorted(must | {int(t) for t in extra}), dtype=np.int64)
+
+
+def test_long_document_reuse_every_tuple_sampled_rows():
+    # 70B-shaped long-document reuse at full size: every one of the 32 tuples, every query head, a seeded quarter of
+    # the suffix rows (first, last and page-boundary rows always) against the oracle's definition on the tuple's
+    # full K/V, which come from the input generator and not from the pool.
+    w = synth.WORKLOADS["long_doc_70b"]
+    wl = DeviceWorkload(w)
+    wl.extend(); torch.cuda.synchronize()
+    assert kvattn.kv_last_async_status(wl.pool) == kvattn.KV_OK
+    e, g = wl.ext, wl.geom
+    G = g.group
+    cu = e.cu_q.cpu().numpy()
+    worst = [0.0, 0.0, 0.0]
+    checked = 0
+    for i in range(len(e.prefix)):
+        P, E = e.prefix[i], e.extend[i]
+        t = _row_sample(P, E, seed=5000 + i)
+        kb, vb = wl.source_kv("ext", i)
+        kf, vf = orc.widen(kb), orc.widen(vb)
+        idx = torch.from_numpy(int(cu[i]) + t).to("cuda")
+        qf = orc.widen(synth.bf16_bits(e.q.index_select(0, idx)))                    # [n][Hq][D]
+        og = e.out.index_select(0, idx).float().cpu().numpy().astype(np.float64)
+        lg = e.lse.index_select(0, idx).cpu().numpy().astype(np.float64)
+        visible = P + t + 1
+        for kvh in range(g.n_kv_heads):
+            hs = slice(kvh * G, (kvh + 1) * G)
+            o, l = orc.attention_rows(qf[:, hs, :].reshape(-1, g.head_dim), kf[:, kvh, :], vf[:, kvh, :],
+                                      np.repeat(visible, G), g.scale)
+            o, l = o.reshape(len(t), G, g.head_dim), l.reshape(len(t), G)
+            worst = [max(worst[0], float(np.max(np.abs(og[:, hs] - o)))), max(worst[1], float(np.max(np.abs(lg[:, hs] - l)))),
+                     max(worst[2], tight_ok(og[:, hs], o))]
+        checked += len(t)
+    assert checked >= 0.25 * e.total_q
+    assert worst[0] <= O_TOL and worst[1] <= LSE_TOL and worst[2] <= 1.0, worst
+    wl.close()
+
+
+def test_pipeline_loop_full_size_eight_steps_with_appends_and_churn():
+    # The two-operator pipeline step as the configuration states it: 48 extend + 192 decode sequences, per step one
+    # kv_append of the new tokens (the suffixes and one token per decode sequence), attn_mixed, then 20 % of the live
+    # pages evicted (poisoned), re-allocated and re-filled; 8 steps, decode contexts growing by one.  Outputs must not
+    # change by a bit across the churn, and a sample of sequences is checked against the oracle every step.
+    w = synth.WORKLOADS["pipeline_step"]
+    steps = 8
+    loop = PipelineLoop(w, steps=steps, poison=True)
+    g = w.geom
+    moved_total = 0
+    for step in range(steps):
+        loop.begin_step()
+        assert loop.step_new_tokens() == sum(loop.extend) + 192
+        loop.append_new()
+        loop.mixed()
+        torch.cuda.synchronize()
+        loop.commit_new()
+        assert kvattn.kv_last_async_status(loop.pool) == kvattn.KV_OK
+        before = [t.clone() for t in (loop.out_ext, loop.lse_ext, loop.out_dec, loop.lse_dec)]
+        assert all(torch.isfinite(t.float()).all() for t in before)
+        # ---- oracle on a sample: the shortest, the longest and one seeded extend tuple; four decode sequences
+        L = [p + e for p, e in zip(loop.prefix, loop.extend)]
+        ext_pick = sorted({int(np.argmin(L)), int(np.argmax(L)), (7 * step + 3) % loop.n_ext})
+        dec_pick = sorted({int(np.argmin(loop.ctx)), int(np.argmax(loop.ctx)), (11 * step + 5) % loop.n_dec,
+                           (29 * step + 1) % loop.n_dec})
+        cu = loop.cu_q.cpu().numpy()
+        for i in ext_pick:
+            kb, vb = loop.source_bits(i)
+            rows = list(range(synth.pages_needed(L[i], 16)))
+            host = orc.PagePool(len(rows), 16, g.n_kv_heads, g.head_dim)
+            host.append(rows, 0, kb, vb)
+            r0, r1 = int(cu[i]), int(cu[i + 1])
+            o, l = orc.attn_extend(host, synth.bf16_bits(loop.q_ext[r0:r1]), g.n_q_heads, [0, r1 - r0],
+                                   synth.block_table([rows]), [loop.prefix[i]], [loop.extend[i]], g.scale)
+            og = loop.out_ext[r0:r1].float().cpu().numpy().astype(np.float64)
+            lg = loop.lse_ext[r0:r1].cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(og - o)) <= O_TOL and np.max(np.abs(lg - l)) <= LSE_TOL and tight_ok(og, o) <= 1.0, (step, i)
+        for j in dec_pick:
+            kb, vb = loop.source_bits(loop.n_ext + j)
+            assert kb.shape[0] == loop.ctx[j]
+            rows = list(range(synth.pages_needed(loop.ctx[j], 16)))
+            host = orc.PagePool(len(rows), 16, g.n_kv_heads, g.head_dim)
+            host.append(rows, 0, kb, vb)
+            o, l = orc.attn_decode(host, synth.bf16_bits(loop.q_dec[j:j + 1]), g.n_q_heads, synth.block_table([rows]),
+                                   [loop.ctx[j]], g.scale)
+            og = loop.out_dec[j:j + 1].float().cpu().numpy().astype(np.float64)
+            lg = loop.lse_dec[j:j + 1].cpu().numpy().astype(np.float64)
+            assert np.max(np.abs(og - o)) <= O_TOL and np.max(np.abs(lg - l)) <= LSE_TOL and tight_ok(og, o) <= 1.0, (step, j)
+        # ---- churn, then the same step again: not a bit may change
+        live = len(loop.live_blocks())
+        moved = loop.churn(0.2)
+        assert moved == int(0.2 * live) and moved > 5000
+        moved_total += moved
+        loop.mixed()
+        torch.cuda.synchronize()
+        after = (loop.out_ext, loop.lse_ext, loop.out_dec, loop.lse_dec)
+        for a_, b_ in zip(before, after):
+            assert torch.equal(a_.view(torch.int32) if a_.dtype == torch.float32 else a_.view(torch.int16),
+                               b_.view(torch.int32) if b_.dtype == torch.float32 else b_.view(torch.int16)), step
+        # the pages really hold the source bits where the tables now say (one moved row, through kv_gather)
+        r = loop.n_ext + dec_pick[0]
+        n = loop.ctx[dec_pick[0]]
+        kk = torch.empty((n, g.n_kv_heads, g.head_dim), dtype=torch.bfloat16, device="cuda")
+        vv = torch.empty_like(kk)
+        kvattn.kv_gather(loop.pool, loop.bt[r].contiguous(), n, kk, vv)
+        torch.cuda.synchronize()
+        kb, vb = loop.source_bits(r)
+        assert np.array_equal(synth.bf16_bits(kk), kb) and np.array_equal(synth.bf16_bits(vv), vb)
+        assert kvattn.kv_last_async_status(loop.pool) == kvattn.KV_OK
+        loop.end_step()
+    _, used, evicted = kvattn.kv_pool_stats(loop.pool)
+    assert evicted == moved_total
+    assert used == sum(len(r) for r in loop.rows)
+    loop.close()

@@ -1,11 +1,12 @@
-"""Seeded random shapes: the tensor-core extend kernel against the small-tile kernel (itself checked against the
-oracle elsewhere) on the same device pool, and the two ways attn_extend_shared can run against each other."""
+"""Seeded random batch shapes: the tensor-core extend kernel and the small-tile kernel on the same device pool, each
+against the oracle and against each other; the two ways attn_extend_shared can run, likewise."""
 import numpy as np
 import pytest
 import torch
 
 from paper_2607_23815_b200 import kvattn, synth
-from harness import Batch, DualPool, LSE_TOL, O_TOL, run_extend
+from oracle import paged_attention as orc
+from harness import Batch, DualPool, LSE_TOL, O_TOL, assert_close, run_extend
 
 pytestmark = pytest.mark.gpu
 GEOMS = [(32, 8, 128), (8, 8, 128), (16, 8, 64), (8, 1, 128), (4, 2, 64), (64, 8, 128)]
@@ -30,13 +31,15 @@ def test_random_batches_tensor_core_vs_small_tile(seed):
     if sum(E) == 0:
         E[0] = 1
     pages = sum(synth.pages_needed(p + e, 16) for p, e in zip(P, E)) + 4
-    dp = DualPool(geom, pages, seed=4100 + seed, with_oracle=False)
+    dp = DualPool(geom, pages, seed=4100 + seed)
     b = Batch(dp, [p + e for p, e in zip(P, E)])
     b.write([(i, 0, P[i] + E[i]) for i in range(B)])
-    tc = run_extend(dp, b, P, E, impl=2, oracle=False)
+    tc = run_extend(dp, b, P, E, impl=2)
     assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+    assert_close(tc, f"random batch {seed}, tensor-core kernel")
     small = run_extend(dp, b, P, E, impl=1, oracle=False)
-    assert not np.isnan(tc["o"]).any()
+    small["o_ref"], small["lse_ref"] = tc["o_ref"], tc["lse_ref"]
+    assert_close(small, f"random batch {seed}, small-tile kernel")
     assert np.max(np.abs(tc["o"] - small["o"])) <= O_TOL
     assert np.max(np.abs(tc["lse"] - small["lse"])) <= LSE_TOL
     dp.close()
@@ -57,7 +60,7 @@ def test_random_fan_outs_one_kernel_vs_three(seed):
     if sum(child_lens) == 0:
         child_lens[0] = 2
     pages = sum(synth.pages_needed(L, 16) for L in parent_lens + child_lens) + 8
-    dp = DualPool(geom, pages, seed=4300 + seed, with_oracle=False)
+    dp = DualPool(geom, pages, seed=4300 + seed)
     parents = Batch(dp, parent_lens, uid0=0)
     parents.write([(g, 0, parent_lens[g]) for g in range(n_par)])
     children = Batch(dp, child_lens, uid0=1000)
@@ -83,6 +86,11 @@ def test_random_fan_outs_one_kernel_vs_three(seed):
         torch.cuda.synchronize()
         assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
         res[impl] = (out.float().cpu().numpy(), lse.cpu().numpy())
+    o_ref, l_ref = orc.attn_extend_shared(dp.host, synth.bf16_bits(q), hq, cu_q, cu_children, parents.block_tables(),
+                                          parent_lens, children.block_tables(), child_lens, geom.scale)
+    for impl in (1, 2):
+        assert_close({"o": res[impl][0].astype(np.float64), "lse": res[impl][1].astype(np.float64), "o_ref": o_ref,
+                      "lse_ref": l_ref}, f"random fan-out {seed}, impl {impl}")
     assert not np.isnan(res[2][0]).any() and not np.isnan(res[1][0]).any()
     assert np.max(np.abs(res[2][0] - res[1][0])) <= O_TOL
     assert np.max(np.abs(res[2][1] - res[1][1])) <= LSE_TOL
