@@ -172,6 +172,19 @@ kv_status_t attn_extend(kv_pool_t* pool, const void* q, int n_q_heads, const int
                         int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                         void* workspace, size_t workspace_bytes, void* stream);
 
+/* kv_append of the suffix and attn_extend in one call (Section 2.1: the downstream operator's prefill both
+ * stores the suffix tokens' K/V and attends with them): k_new / v_new [dev] bf16 [total_q][n_kv_heads][head_dim],
+ * ragged by cu_q like q, are written to positions prefix_lens[i] .. prefix_lens[i]+extend_lens[i]-1 of sequence
+ * i's pages exactly as kv_append(k_new, v_new, cu_q, prefix_lens, NULL, block_tables, ...) would (same bits, same
+ * clearing of the last page's tail), then the suffix attends exactly as attn_extend would (same bits).  What it
+ * saves is launches: the rows are scattered by the kernel that also prepares the attention kernel's work list, and
+ * the attention kernel is launched so that its start-up overlaps that kernel.  Arguments, workspace and errors as
+ * for kv_append and attn_extend. */
+kv_status_t attn_extend_append(kv_pool_t* pool, const void* q, const void* k_new, const void* v_new, int n_q_heads,
+                               const int* cu_q, const int* block_tables, int max_pages, const int* prefix_lens,
+                               const int* extend_lens, int batch, int total_q, int max_extend_len, int max_total_len,
+                               float scale, void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream);
+
 /* One pipeline step from host memory: the call for a caller whose suffix Q/K/V, lengths and block tables live
  * in host buffers (pinned, if the call is to return before the copies are done).  On the given stream it
  * copies the inputs into `staging` [dev], appends the suffix K/V rows of sequence i at positions

@@ -1,4 +1,5 @@
 // Public attention entry points: argument checks, kernel selection, the mixed-batch launcher.
+#include "append.cuh"
 #include "common.cuh"
 
 namespace kvattn {
@@ -16,7 +17,7 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                              void* workspace, size_t workspace_bytes, int cta_cap, int mode, const FanArgs* fan,
-                             cudaStream_t st);
+                             const AppendArgs* app, cudaStream_t st);
 
 size_t extend_shared_workspace_bytes(const kv_pool_t* p, int n_q_heads, int n_parents, int n_children, int total_q,
                                      int max_parent_len);
@@ -59,10 +60,13 @@ size_t attn_workspace_bytes(const kv_pool_t* p, int n_q_heads, int batch_ext, in
          align256(decode_workspace_bytes(n_q_heads, p->head_dim, batch_dec, max_ctx_len)) + 256;
 }
 
+// k_new / v_new non-null: the suffix K/V rows (ragged by cu_q like Q) are first written to positions prefix_lens[i] ..
+// of their sequences' pages, in the kernel that also builds the attention kernel's plan.
 static kv_status_t extend_impl(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                                int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                                int max_extend_len, int max_total_len, float scale, void* out, float* lse,
-                               void* workspace, size_t workspace_bytes, int cta_cap, void* stream) {
+                               void* workspace, size_t workspace_bytes, int cta_cap, void* stream,
+                               const void* k_new = nullptr, const void* v_new = nullptr) {
   if (p == nullptr || batch < 0 || total_q < 0 || max_pages < 0 || max_extend_len < 0 || max_total_len < 0)
     return KV_ERR_INVALID;
   if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
@@ -77,9 +81,15 @@ static kv_status_t extend_impl(kv_pool_t* p, const void* q, int n_q_heads, const
   const bool tc_ok = extend_tc_supported(p, n_q_heads) && scale > 0.f;  // the tensor-core kernel folds a positive scale into the row maximum
   if (impl == 2 && !tc_ok) return KV_ERR_UNSUPPORTED;
   if (impl == 2 || (impl == 0 && tc_ok)) {
+    const AppendArgs app{(const uint4*)k_new, (const uint4*)v_new, cu_q, prefix_lens, nullptr, block_tables, max_pages, batch,
+                         total_q};
     return launch_extend_tc(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
                             max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, cta_cap, 0,
-                            nullptr, (cudaStream_t)stream);
+                            nullptr, k_new != nullptr ? &app : nullptr, (cudaStream_t)stream);
+  }
+  if (k_new != nullptr) {  // the small-tile kernel has no plan to share a launch with: append, then attend
+    const kv_status_t as = kv_append(p, k_new, v_new, cu_q, prefix_lens, nullptr, block_tables, max_pages, batch, total_q, stream);
+    if (as != KV_OK) return as;
   }
   return launch_extend_small(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch,
                              max_extend_len, max_total_len, scale, out, lse, (cudaStream_t)stream);
@@ -91,6 +101,18 @@ kv_status_t attn_extend(kv_pool_t* p, const void* q, int n_q_heads, const int* c
                         size_t workspace_bytes, void* stream) {
   return extend_impl(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
                      max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, 0, stream);
+}
+
+kv_status_t attn_extend_append(kv_pool_t* p, const void* q, const void* k_new, const void* v_new, int n_q_heads,
+                               const int* cu_q, const int* block_tables, int max_pages, const int* prefix_lens,
+                               const int* extend_lens, int batch, int total_q, int max_extend_len, int max_total_len,
+                               float scale, void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream) {
+  if (p != nullptr && batch > 0 && total_q > 0) {
+    if (k_new == nullptr || v_new == nullptr) return KV_ERR_INVALID;
+    if ((((uintptr_t)k_new) | ((uintptr_t)v_new)) & 15) return KV_ERR_INVALID;
+  }
+  return extend_impl(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
+                     max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, 0, stream, k_new, v_new);
 }
 
 size_t attn_extend_shared_workspace_bytes(const kv_pool_t* p, int n_q_heads, int n_parents, int n_children, int total_q,
@@ -208,10 +230,9 @@ kv_status_t attn_extend_host(kv_pool_t* p, const void* q, const void* k_new, con
   const int* d_pl = reinterpret_cast<const int*>(d + L.pl);
   const int* d_el = reinterpret_cast<const int*>(d + L.el);
   // the suffix K/V rows of sequence i go to positions prefix_lens[i] .. of its pages, then the suffix attends
-  kv_status_t s = kv_append(p, d + L.k, d + L.v, d_cu, d_pl, nullptr, d_bt, max_pages, batch, total_q, stream);
-  if (s == KV_OK)
-    s = attn_extend(p, d + L.q, n_q_heads, d_cu, d_bt, max_pages, d_pl, d_el, batch, total_q, max_extend_len,
-                    max_total_len, scale, d + L.out, reinterpret_cast<float*>(d + L.lse), d + L.ws, L.total - L.ws, stream);
+  kv_status_t s = attn_extend_append(p, d + L.q, d + L.k, d + L.v, n_q_heads, d_cu, d_bt, max_pages, d_pl, d_el, batch, total_q,
+                                     max_extend_len, max_total_len, scale, d + L.out, reinterpret_cast<float*>(d + L.lse),
+                                     d + L.ws, L.total - L.ws, stream);
   KV_CUDA_OK(cudaEventRecord(hs->ran, st));
   if (s != KV_OK) return s;
   KV_CUDA_OK(cudaStreamWaitEvent(p->d2h_stream, hs->ran, 0));
@@ -271,7 +292,7 @@ kv_status_t attn_mixed(kv_pool_t* p, int n_q_heads, float scale, const attn_exte
     KV_CUDA_OK(cudaStreamWaitEvent(p->side_stream, p->ev_fork, 0));
     kv_status_t s = extend_impl(p, ext->q, n_q_heads, ext->cu_q, ext->block_tables, ext->max_pages, ext->prefix_lens,
                                 ext->extend_lens, ext->batch, ext->total_q, ext->max_extend_len, ext->max_total_len,
-                                scale, ext->out, ext->lse, ws, ext_bytes, g_mixed_extend_ctas.load(), st);
+                                scale, ext->out, ext->lse, ws, ext_bytes, g_mixed_extend_ctas.load() > 0 ? g_mixed_extend_ctas.load() : -1, st);
     kv_status_t s2 = KV_OK;
     if (s == KV_OK)
       s2 = attn_decode(p, dec->q, n_q_heads, dec->block_tables, dec->max_pages, dec->ctx_lens, dec->batch,

@@ -26,6 +26,7 @@
 // tensor memory and returns.
 #include <cuda.h>  // CUtensorMap and its enums (types only: the encoder is looked up at run time)
 
+#include "append.cuh"
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -130,14 +131,32 @@ __device__ __forceinline__ ItemRec make_item(int seq, int tp, int P, int E, int 
   return r;
 }
 
-__global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restrict__ prefix_lens,
-                                                              const int* __restrict__ extend_lens,
-                                                              const int* __restrict__ cu_q, int batch, int max_tp,
-                                                              int lg, int max_steps, int capacity, int max_pages,
-                                                              int mode, FanArgs fan, int groups,
-                                                              int* status, int4* __restrict__ items,
-                                                              int* __restrict__ n_items, int* __restrict__ next_item,
-                                                              int first_free_item) {
+struct PlanArgs {
+  const int* prefix_lens;
+  const int* extend_lens;
+  const int* cu_q;
+  int batch, max_tp, lg, max_steps, capacity, max_pages, mode;
+  FanArgs fan;
+  int groups;
+  int* status;
+  int4* items;
+  int* n_items;
+  int* next_item;
+  int first_free_item;
+};
+
+// Runs in one block of 1024 threads.
+__device__ __forceinline__ void plan_body(const PlanArgs& pa) {
+  const int* __restrict__ prefix_lens = pa.prefix_lens;
+  const int* __restrict__ extend_lens = pa.extend_lens;
+  const int* __restrict__ cu_q = pa.cu_q;
+  const int batch = pa.batch, max_tp = pa.max_tp, lg = pa.lg, max_steps = pa.max_steps, capacity = pa.capacity;
+  const int max_pages = pa.max_pages, mode = pa.mode, groups = pa.groups, first_free_item = pa.first_free_item;
+  const FanArgs& fan = pa.fan;
+  int* status = pa.status;
+  int4* __restrict__ items = pa.items;
+  int* __restrict__ n_items = pa.n_items;
+  int* __restrict__ next_item = pa.next_item;
   if (threadIdx.x == 0) *next_item = first_free_item;  // the CTAs start on items 0 .. grid-1 without asking
   __shared__ int hist[kPlanBuckets];
   for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
@@ -268,6 +287,24 @@ __global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const int* __restr
   }
 }
 
+__global__ void __launch_bounds__(1024) extend_tc_plan_kernel(const PlanArgs pa) {
+  launch_dependents();  // the attention kernel may set itself up meanwhile; it waits for this kernel before it reads the plan
+  plan_body(pa);
+}
+
+// Prologue of the fused append + extend call: block 0 builds the plan while the other blocks scatter the suffix K/V
+// rows into their pages (one warp per token), so the step has one small kernel in front of the attention kernel
+// instead of two in a row, and the attention kernel's launch and set-up overlap it.
+__global__ void __launch_bounds__(1024) extend_prologue_kernel(const PlanArgs pa, const PoolView pool, const AppendArgs ap) {
+  launch_dependents();
+  if (blockIdx.x == 0) {
+    plan_body(pa);
+  } else {
+    const int warps_per_block = blockDim.x >> 5;
+    append_tokens<4>(pool, ap, (blockIdx.x - 1) * warps_per_block + (threadIdx.x >> 5), (gridDim.x - 1) * warps_per_block);
+  }
+}
+
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float d;
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -345,7 +382,7 @@ __device__ __forceinline__ bool fetch_item(const TcArgs& a, int k, int n_total, 
   if (k >= n_total) return false;
   const int Hkv = a.pool.n_kv_heads;
   const int e = k / Hkv;
-  const int4 r0 = __ldg(a.items + 2 * e), r1 = __ldg(a.items + 2 * e + 1);
+  const int4 r0 = __ldcg(a.items + 2 * e), r1 = __ldcg(a.items + 2 * e + 1);  // written by the kernel before this one: read through L2
   it.seq = r0.x; it.tp = r0.y; it.P = r0.z; it.E = r0.w;
   it.row0 = r1.x; it.n_kv[0] = r1.y; it.n_kv[1] = r1.z; it.kv_end = r1.w;
   it.c_first = 0;
@@ -431,7 +468,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = sm.tmem_base;
-  const int n_total = __ldg(a.n_items) * a.pool.n_kv_heads;
+  // Everything up to here touched only this CTA's own shared and tensor memory and may have run while the kernel in
+  // front of this one (the plan, or the plan and the suffix append) was still at work; its results are needed now.
+  dependency_wait();
+  const int n_total = __ldcg(a.n_items) * a.pool.n_kv_heads;
   const int Hkv = a.pool.n_kv_heads;
   // Round r of this CTA works on item sched_get(r) of the global list (>= n_total: no more work).  A warp
   // calls sched_release(r) once it no longer needs the slot.
@@ -1040,13 +1080,14 @@ static kv_status_t make_q_map(CUtensorMap* map, const void* q, int total_q, int 
 static kv_status_t tc_grid(const kv_pool_t* p, int n_items_bound, int cta_cap, int* grid_out) {
   const int sm_count = sm_count_of(p->device);
   int grid = n_items_bound < sm_count ? (n_items_bound < 1 ? 1 : n_items_bound) : sm_count;
-  if (cta_cap > 0 && grid > cta_cap) grid = cta_cap;  // leave the other SMs to work that runs beside this kernel
+  if (cta_cap > 0 && grid > cta_cap) grid = cta_cap;  // leave the other SMs to work that runs beside this kernel (< 0: no
+                                                      // cap, and the kernel is launched without the early start)
   *grid_out = grid;
   return KV_OK;
 }
 
 template <int D, bool OPT>
-static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid, int device, cudaStream_t st) {
+static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid, int device, bool early_start, cudaStream_t st) {
   const size_t smem = sizeof(TcSmem<D>);
   static std::atomic<bool> configured[kMaxDevices];  // the attribute belongs to the function on one device
   if (device < 0 || device >= kMaxDevices) return KV_ERR_INVALID;
@@ -1054,9 +1095,21 @@ static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid
     KV_CUDA_OK(cudaFuncSetAttribute(attn_extend_tc_kernel<D, OPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured[device].store(true, std::memory_order_release);
   }
-  attn_extend_tc_kernel<D, OPT><<<grid, kTcThreads, smem, st>>>(a, q_map);
+  // early_start: launched so that it may start while the plan kernel in front of it still runs (it waits for it
+  // inside).  Not wanted when another kernel is meant to take the SMs first (the mixed step's decode kernel): CTAs
+  // that sit on an SM waiting for the plan keep that kernel's blocks away.
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)grid);
+  cfg.blockDim = dim3(kTcThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = early_start ? 1 : 0;
+  KV_CUDA_OK(cudaLaunchKernelEx(&cfg, attn_extend_tc_kernel<D, OPT>, a, q_map));
   count_launch();
-  KV_CUDA_OK(cudaGetLastError());
   return KV_OK;
 }
 
@@ -1064,7 +1117,7 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                              void* workspace, size_t workspace_bytes, int cta_cap, int mode, const FanArgs* fan,
-                             cudaStream_t st) {
+                             const AppendArgs* app, cudaStream_t st) {
   const size_t need = extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch, total_q, max_total_len);
   if (workspace == nullptr || workspace_bytes < need) return KV_ERR_WORKSPACE;
   const int G = n_q_heads / p->n_kv_heads;
@@ -1096,9 +1149,17 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   groups = groups < 1 ? 1 : groups;
   groups = groups > batch ? batch : groups;
   groups = groups > kPlanBuckets / 16 ? kPlanBuckets / 16 : groups;
-  extend_tc_plan_kernel<<<1, 1024, 0, st>>>(prefix_lens, extend_lens, cu_q, batch, max_tp, lg, max_steps, (int)capacity,
-                                            max_pages, mode, fan != nullptr ? *fan : FanArgs{}, groups, p->d_status, items,
-                                            n_items, n_items + 1, grid);
+  const PlanArgs pa{prefix_lens, extend_lens, cu_q, batch, max_tp, lg, max_steps, (int)capacity, max_pages, mode,
+                    fan != nullptr ? *fan : FanArgs{}, groups, p->d_status, items, n_items, n_items + 1, grid};
+  if (app != nullptr && app->total_new > 0) {
+    // plan block + append blocks (32 warps each, one warp per token, all blocks resident at once)
+    const int64_t want = ((int64_t)app->total_new + 31) / 32;
+    const int64_t cap = 2 * (int64_t)sm_count_of(p->device) - 1;
+    const int blocks = (int)(want < cap ? want : cap);
+    extend_prologue_kernel<<<1 + blocks, 1024, 0, st>>>(pa, p->view(), *app);
+  } else {
+    extend_tc_plan_kernel<<<1, 1024, 0, st>>>(pa);
+  }
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
 
@@ -1125,9 +1186,10 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   // Skipping the search for the row maximum pays where items have many KV steps (measured: +2 % on the
   // long-document shapes, -1 % on the 8B extend batch whose items have a dozen steps)
   const bool opt = max_total_len >= kOptimisticMinLen;
+  const bool early = cta_cap >= 0;
   if (p->head_dim == 128)
-    return opt ? launch_tc<128, true>(a, q_map, grid, p->device, st) : launch_tc<128, false>(a, q_map, grid, p->device, st);
-  return opt ? launch_tc<64, true>(a, q_map, grid, p->device, st) : launch_tc<64, false>(a, q_map, grid, p->device, st);
+    return opt ? launch_tc<128, true>(a, q_map, grid, p->device, early, st) : launch_tc<128, false>(a, q_map, grid, p->device, early, st);
+  return opt ? launch_tc<64, true>(a, q_map, grid, p->device, early, st) : launch_tc<64, false>(a, q_map, grid, p->device, early, st);
 }
 
 }  // namespace kvattn

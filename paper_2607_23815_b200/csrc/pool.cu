@@ -3,6 +3,7 @@
 #include <new>
 
 #include "common.cuh"
+#include "append.cuh"
 
 namespace kvattn {
 
@@ -13,75 +14,8 @@ std::atomic<int64_t> g_launches{0};
 // rows (coalesced loads, all in flight before the first store); the eight chunks of a 64-dim half land,
 // permuted, in one 128-byte row of the page (full-line 16-byte stores).
 // ------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) append_kernel(PoolView pool, const uint4* __restrict__ k_new,
-                                                     const uint4* __restrict__ v_new,
-                                                     const int* __restrict__ cu_new,
-                                                     const int* __restrict__ start_pos,
-                                                     const int* __restrict__ seg_row,
-                                                     const int* __restrict__ block_tables, int max_pages,
-                                                     int n_segments, int total_new) {
-  // One warp per token: the token's segment, position and page are looked up once, then the lanes copy the
-  // token's 16-byte chunks (n_kv_heads * head_dim / 8 of them), all loads of a token in flight before its stores.
-  const int chunks_per_row = pool.head_dim >> 3;               // 16-byte chunks per (token, head)
-  const int chunks_per_token = pool.n_kv_heads * chunks_per_row;
-  const size_t blk = block_bytes(pool.head_dim);
-  const int lane = threadIdx.x & 31;
-  const int warps = (gridDim.x * blockDim.x) >> 5;
-  constexpr int kMaxPerLane = 8;                               // chunks a lane holds at once (256 chunks per pass)
-  for (int token = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; token < total_new; token += warps) {
-    // segment of this token: last s with cu_new[s] <= token
-    int lo = 0, hi = n_segments;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (__ldg(cu_new + mid) <= token) lo = mid; else hi = mid;
-    }
-    const int seg = lo;
-    const int seg_begin = __ldg(cu_new + seg), seg_end = __ldg(cu_new + seg + 1);
-    if (token >= seg_end) continue;                            // cu_new not covering this row: skip
-    const int pos = __ldg(start_pos + seg) + (token - seg_begin);
-    const int row = seg_row ? __ldg(seg_row + seg) : seg;
-    const int blk_idx = pos >> 4;
-    if (pos < 0 || blk_idx >= max_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
-    const int page = __ldg(block_tables + (int64_t)row * max_pages + blk_idx);
-    if (page < 0 || page >= pool.num_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
-    const size_t page_off = (size_t)page * pool.n_kv_heads * blk;
-    const uint4* ksrc = k_new + (int64_t)token * chunks_per_token;
-    const uint4* vsrc = v_new + (int64_t)token * chunks_per_token;
-    const bool last = token + 1 == seg_end;
-    for (int c0 = 0; c0 < chunks_per_token; c0 += 32 * kMaxPerLane) {
-      uint4 kk[kMaxPerLane], vv[kMaxPerLane];
-#pragma unroll
-      for (int i = 0; i < kMaxPerLane; ++i) {
-        const int c = c0 + i * 32 + lane;
-        if (c < chunks_per_token) {
-          kk[i] = __ldg(ksrc + c);
-          vv[i] = __ldg(vsrc + c);
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < kMaxPerLane; ++i) {
-        const int c = c0 + i * 32 + lane;
-        if (c < chunks_per_token) {
-          const int head = c / chunks_per_row, dchunk = c - head * chunks_per_row;
-          const size_t blk_off = page_off + (size_t)head * blk;
-          const size_t off = blk_off + chunk_offset_bytes(pos & 15, dchunk, pool.head_dim);
-          *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + off) = kk[i];
-          *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + off) = vv[i];
-          // The segment's last token also clears the slots behind it in its page.  Slots past a sequence's
-          // end therefore never hold NaN/Inf bit patterns, which the tensor-core kernel relies on: it
-          // multiplies those V rows by probabilities that are exactly 0.
-          if (last) {
-            const uint4 z = make_uint4(0, 0, 0, 0);
-            for (int slot = (pos & 15) + 1; slot < kPageSize; ++slot) {
-              const size_t o2 = blk_off + chunk_offset_bytes(slot, dchunk, pool.head_dim);
-              *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.k) + o2) = z;
-              *reinterpret_cast<uint4*>(reinterpret_cast<char*>(pool.v) + o2) = z;
-            }
-          }
-        }
-      }
-    }
-  }
+__global__ void __launch_bounds__(256) append_kernel(PoolView pool, AppendArgs a) {
+  append_tokens<8>(pool, a, (blockIdx.x * blockDim.x + threadIdx.x) >> 5, (gridDim.x * blockDim.x) >> 5);
 }
 
 __global__ void __launch_bounds__(256) gather_kernel(PoolView pool, const int* __restrict__ block_row, int len,
@@ -453,9 +387,9 @@ kv_status_t kv_append(kv_pool_t* p, const void* k_new, const void* v_new, const 
     return KV_ERR_INVALID;
   if ((((uintptr_t)k_new) | ((uintptr_t)v_new)) & 15) return KV_ERR_INVALID;
   if (!on_pool_device(p)) return KV_ERR_INVALID;
-  append_kernel<<<grid_for(p, (int64_t)total_new * 32, 256), 256, 0, (cudaStream_t)stream>>>(  // one warp per token
-      p->view(), (const uint4*)k_new, (const uint4*)v_new, cu_new, start_pos, seg_row, block_tables, max_pages,
-      n_segments, total_new);
+  const AppendArgs a{(const uint4*)k_new, (const uint4*)v_new, cu_new, start_pos, seg_row, block_tables, max_pages, n_segments,
+                     total_new};
+  append_kernel<<<grid_for(p, (int64_t)total_new * 32, 256), 256, 0, (cudaStream_t)stream>>>(p->view(), a);  // one warp per token
   count_launch();
   KV_CUDA_OK(cudaGetLastError());
   return KV_OK;

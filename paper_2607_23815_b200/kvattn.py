@@ -61,6 +61,7 @@ _SIGNATURES = {
     "kv_gather": (_I, [_P, _P, _I, _P, _P, _P]),
     "attn_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I, _I]),
     "attn_extend": (_I, [_P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
+    "attn_extend_append": (_I, [_P, _P, _P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_extend_host_staging_bytes": (_SZ, [_P, _I, _I, _I, _I, _I]),
     "attn_extend_host": (_I, [_P, _P, _P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_extend_shared_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I]),
@@ -256,6 +257,17 @@ def attn_extend(pool: Pool, q, cu_q, block_tables, prefix_lens, extend_lens, max
                              _dev_ptr(out), _dev_ptr(lse), _dev_ptr(workspace),
                              0 if workspace is None else workspace.numel() * workspace.element_size(),
                              _stream(stream)), "attn_extend")
+
+
+def attn_extend_append(pool: Pool, q, k_new, v_new, cu_q, block_tables, prefix_lens, extend_lens, max_extend_len,
+                       max_total_len, scale, out, lse, workspace=None, stream=None):
+    """kv_append of the suffix rows (k_new, v_new, ragged by cu_q) at positions prefix_lens[i].. and attn_extend, one call."""
+    _check(lib().attn_extend_append(pool.handle, _dev_ptr(q), _dev_ptr(k_new), _dev_ptr(v_new), q.shape[1], _dev_ptr(cu_q),
+                                    _dev_ptr(block_tables), block_tables.shape[1], _dev_ptr(prefix_lens),
+                                    _dev_ptr(extend_lens), prefix_lens.numel(), q.shape[0], max_extend_len, max_total_len,
+                                    float(scale), _dev_ptr(out), _dev_ptr(lse), _dev_ptr(workspace),
+                                    0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                    _stream(stream)), "attn_extend_append")
 
 
 def attn_extend_host_staging_bytes(pool: Pool, n_q_heads, batch, total_q, max_pages, max_total_len) -> int:

@@ -165,6 +165,12 @@ class DeviceWorkload:
         kvattn.attn_extend(self.pool, e.q, e.cu_q, e.block_tables, e.prefix_lens, e.extend_lens, e.max_extend,
                            e.max_total, self.geom.scale, e.out, e.lse, self.workspace, stream)
 
+    def extend_append(self, stream=None):
+        """The downstream operator's prefill as one call: the suffix K/V rows go into their pages and the suffix attends."""
+        e = self.ext
+        kvattn.attn_extend_append(self.pool, e.q, e.k_new, e.v_new, e.cu_q, e.block_tables, e.prefix_lens, e.extend_lens,
+                                  e.max_extend, e.max_total, self.geom.scale, e.out, e.lse, self.workspace, stream)
+
     def decode(self, stream=None):
         d = self.dec
         kvattn.attn_decode(self.pool, d.q, d.block_tables, d.ctx_lens, d.max_ctx, self.geom.scale, d.out, d.lse,

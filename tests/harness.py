@@ -33,6 +33,7 @@ class DualPool:
     def __init__(self, geom: synth.Geometry, num_pages: int, seed: int, device="cuda", fill=NAN_BITS,
                  with_oracle=True):
         self.geom, self.num_pages, self.seed, self.device = geom, num_pages, seed, device
+        self.gen_device = device        # where the input generator runs ("cpu": no generator kernels on the GPU)
         n_elem = num_pages * geom.n_kv_heads * geom.page_size * geom.head_dim
         # caller-owned buffers, pre-filled (NaN by default) so that any stale read shows up
         self.k_buf = torch.full((n_elem,), fill, dtype=torch.int16, device=device)
@@ -102,13 +103,14 @@ class Batch:
 
     def kv(self, i: int, lo: int, hi: int):
         g, dp = self.dp.geom, self.dp
-        k = synth.normal_bf16(dp.seed, synth.TAG_K, self.uids[i], lo, hi - lo, g.n_kv_heads, g.head_dim, dp.device)
-        v = synth.normal_bf16(dp.seed, synth.TAG_V, self.uids[i], lo, hi - lo, g.n_kv_heads, g.head_dim, dp.device)
-        return k, v
+        k = synth.normal_bf16(dp.seed, synth.TAG_K, self.uids[i], lo, hi - lo, g.n_kv_heads, g.head_dim, dp.gen_device)
+        v = synth.normal_bf16(dp.seed, synth.TAG_V, self.uids[i], lo, hi - lo, g.n_kv_heads, g.head_dim, dp.gen_device)
+        return k.to(dp.device), v.to(dp.device)
 
     def q(self, i: int, lo: int, hi: int):
         g, dp = self.dp.geom, self.dp
-        return synth.normal_bf16(dp.seed, synth.TAG_Q, self.uids[i], lo, hi - lo, g.n_q_heads, g.head_dim, dp.device)
+        return synth.normal_bf16(dp.seed, synth.TAG_Q, self.uids[i], lo, hi - lo, g.n_q_heads, g.head_dim,
+                                 dp.gen_device).to(dp.device)
 
     def write(self, ranges):
         """ranges: list of (seq index, lo, hi): append tokens lo..hi-1 of those sequences."""

@@ -238,3 +238,49 @@ def test_more_sequences_than_the_plan_ranks():
         assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
         assert_close(res, f"{n} sequences")
         dp.close()
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+@pytest.mark.parametrize("hq,hkv,d", [(32, 8, 128), (4, 2, 64)])
+def test_append_and_extend_in_one_call_is_bit_identical_to_the_two_calls(impl, hq, hkv, d):
+    # attn_extend_append = kv_append(suffix) + attn_extend with fewer launches: the whole pool image, O and LSE must
+    # come out bit for bit as from the two calls, and O / LSE within tolerance of the oracle.
+    geom = synth.Geometry(hq, hkv, d)
+    _skip_if_no_tc(impl, geom)
+    P = [0, 17, 160, 500, 31, 16, 1000]
+    E = [40, 1, 129, 64, 300, 16, 7]
+    L = [p + e for p, e in zip(P, E)]
+    imgs, outs = [], []
+    for fused in (False, True):
+        dp = DualPool(geom, 160, seed=321)
+        b = Batch(dp, L)
+        b.write([(i, 0, P[i]) for i in range(len(P))])                       # the upstream operator's prefix only
+        ks, vs = zip(*[b.kv(i, P[i], L[i]) for i in range(len(P))])
+        if not fused:
+            dp.append(b.rows, [(i, P[i]) for i in range(len(P))], list(ks), list(vs))
+            res = run_extend(dp, b, P, E, impl=impl)
+            assert_close(res, "append then extend")
+        else:
+            q = torch.cat([b.q(i, P[i], L[i]) for i in range(len(P))]).contiguous()
+            k_new, v_new = torch.cat(ks).contiguous(), torch.cat(vs).contiguous()
+            t = lambda x: torch.tensor(np.asarray(x), dtype=torch.int32, device="cuda")
+            out = torch.full_like(q, float("nan"))
+            lse = torch.full((q.shape[0], hq), float("nan"), dtype=torch.float32, device="cuda")
+            ws = torch.empty(kvattn.attn_workspace_bytes(dp.pool, hq, len(P), int(q.shape[0]), max(L), 0, 0), dtype=torch.uint8,
+                             device="cuda")
+            kvattn.kvattn_set_extend_impl(impl)
+            try:
+                kvattn.attn_extend_append(dp.pool, q, k_new, v_new, t(np.concatenate([[0], np.cumsum(E)])),
+                                          torch.from_numpy(b.block_tables()).to("cuda"), t(P), t(E), max(E), max(L), geom.scale,
+                                          out, lse, ws)
+            finally:
+                kvattn.kvattn_set_extend_impl(0)
+            torch.cuda.synchronize()
+            res = {"o_bits": synth.bf16_bits(out), "lse_raw": lse.cpu().numpy().copy()}
+        assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+        imgs.append(dp.device_image())
+        outs.append(res)
+        dp.close()
+    assert np.array_equal(imgs[0][0], imgs[1][0]) and np.array_equal(imgs[0][1], imgs[1][1])   # K and V pool images
+    assert np.array_equal(outs[0]["o_bits"], outs[1]["o_bits"])
+    assert np.array_equal(outs[0]["lse_raw"], outs[1]["lse_raw"])
