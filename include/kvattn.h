@@ -185,6 +185,21 @@ kv_status_t attn_extend_append(kv_pool_t* pool, const void* q, const void* k_new
                                const int* extend_lens, int batch, int total_q, int max_extend_len, int max_total_len,
                                float scale, void* out, float* lse, void* workspace, size_t workspace_bytes, void* stream);
 
+/* The same batch passes through every layer of the model with the same lengths and block tables (Section 2.1: K/V
+ * are kept per layer), so what attn_extend derives from the lengths alone - its list of work items - can be built
+ * once per step and reused by every layer.  attn_extend_plan builds it into the workspace; attn_extend_planned is
+ * attn_extend without that part and must get the arguments (lengths, tables, bounds, workspace) the plan was built
+ * with; the plan stays valid for any number of attn_extend_planned calls, one at a time, until the workspace is
+ * written by another call.  Results are bit-identical to attn_extend.  The pages need not hold the K/V yet when the
+ * plan is built. */
+kv_status_t attn_extend_plan(kv_pool_t* pool, int n_q_heads, const int* cu_q, const int* block_tables, int max_pages,
+                             const int* prefix_lens, const int* extend_lens, int batch, int total_q, int max_extend_len,
+                             int max_total_len, void* workspace, size_t workspace_bytes, void* stream);
+kv_status_t attn_extend_planned(kv_pool_t* pool, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                                int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                                int max_extend_len, int max_total_len, float scale, void* out, float* lse,
+                                void* workspace, size_t workspace_bytes, void* stream);
+
 /* One pipeline step from host memory: the call for a caller whose suffix Q/K/V, lengths and block tables live
  * in host buffers (pinned, if the call is to return before the copies are done).  On the given stream it
  * copies the inputs into `staging` [dev], appends the suffix K/V rows of sequence i at positions

@@ -17,7 +17,7 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                              void* workspace, size_t workspace_bytes, int cta_cap, int mode, const FanArgs* fan,
-                             const AppendArgs* app, cudaStream_t st);
+                             const AppendArgs* app, int phase, cudaStream_t st);
 
 size_t extend_shared_workspace_bytes(const kv_pool_t* p, int n_q_heads, int n_parents, int n_children, int total_q,
                                      int max_parent_len);
@@ -66,26 +66,30 @@ static kv_status_t extend_impl(kv_pool_t* p, const void* q, int n_q_heads, const
                                int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                                int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                                void* workspace, size_t workspace_bytes, int cta_cap, void* stream,
-                               const void* k_new = nullptr, const void* v_new = nullptr) {
+                               const void* k_new = nullptr, const void* v_new = nullptr, int phase = 0) {
   if (p == nullptr || batch < 0 || total_q < 0 || max_pages < 0 || max_extend_len < 0 || max_total_len < 0)
     return KV_ERR_INVALID;
   if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
   if (batch == 0 || total_q == 0 || max_extend_len == 0) return KV_OK;
-  if (q == nullptr || cu_q == nullptr || block_tables == nullptr || prefix_lens == nullptr ||
-      extend_lens == nullptr || out == nullptr || lse == nullptr)
-    return KV_ERR_INVALID;
+  if (cu_q == nullptr || block_tables == nullptr || prefix_lens == nullptr || extend_lens == nullptr) return KV_ERR_INVALID;
+  if (phase != 1 && (q == nullptr || out == nullptr || lse == nullptr)) return KV_ERR_INVALID;
   if ((((uintptr_t)q) | ((uintptr_t)out)) & 15) return KV_ERR_INVALID;
   if (max_total_len < max_extend_len || max_total_len > (int64_t)max_pages * kPageSize) return KV_ERR_INVALID;
   if (!on_pool_device(p)) return KV_ERR_INVALID;
   const int impl = g_extend_impl.load();
   const bool tc_ok = extend_tc_supported(p, n_q_heads) && scale > 0.f;  // the tensor-core kernel folds a positive scale into the row maximum
   if (impl == 2 && !tc_ok) return KV_ERR_UNSUPPORTED;
+  if (phase != 0 && !(impl == 2 || (impl == 0 && tc_ok))) {
+    // the small-tile kernel has no plan: planning is a no-op and the planned call is the plain one
+    if (phase == 1) return KV_OK;
+    phase = 0;
+  }
   if (impl == 2 || (impl == 0 && tc_ok)) {
     const AppendArgs app{(const uint4*)k_new, (const uint4*)v_new, cu_q, prefix_lens, nullptr, block_tables, max_pages, batch,
                          total_q};
     return launch_extend_tc(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
                             max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, cta_cap, 0,
-                            nullptr, k_new != nullptr ? &app : nullptr, (cudaStream_t)stream);
+                            nullptr, k_new != nullptr ? &app : nullptr, phase, (cudaStream_t)stream);
   }
   if (k_new != nullptr) {  // the small-tile kernel has no plan to share a launch with: append, then attend
     const kv_status_t as = kv_append(p, k_new, v_new, cu_q, prefix_lens, nullptr, block_tables, max_pages, batch, total_q, stream);
@@ -113,6 +117,23 @@ kv_status_t attn_extend_append(kv_pool_t* p, const void* q, const void* k_new, c
   }
   return extend_impl(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
                      max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, 0, stream, k_new, v_new);
+}
+
+kv_status_t attn_extend_plan(kv_pool_t* p, int n_q_heads, const int* cu_q, const int* block_tables, int max_pages,
+                             const int* prefix_lens, const int* extend_lens, int batch, int total_q, int max_extend_len,
+                             int max_total_len, void* workspace, size_t workspace_bytes, void* stream) {
+  return extend_impl(p, nullptr, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
+                     max_extend_len, max_total_len, 1.f, nullptr, nullptr, workspace, workspace_bytes, 0, stream, nullptr,
+                     nullptr, 1);
+}
+
+kv_status_t attn_extend_planned(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
+                                int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
+                                int max_extend_len, int max_total_len, float scale, void* out, float* lse,
+                                void* workspace, size_t workspace_bytes, void* stream) {
+  return extend_impl(p, q, n_q_heads, cu_q, block_tables, max_pages, prefix_lens, extend_lens, batch, total_q,
+                     max_extend_len, max_total_len, scale, out, lse, workspace, workspace_bytes, 0, stream, nullptr, nullptr,
+                     2);
 }
 
 size_t attn_extend_shared_workspace_bytes(const kv_pool_t* p, int n_q_heads, int n_parents, int n_children, int total_q,

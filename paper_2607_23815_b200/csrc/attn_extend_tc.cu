@@ -157,7 +157,10 @@ __device__ __forceinline__ void plan_body(const PlanArgs& pa) {
   int4* __restrict__ items = pa.items;
   int* __restrict__ n_items = pa.n_items;
   int* __restrict__ next_item = pa.next_item;
-  if (threadIdx.x == 0) *next_item = first_free_item;  // the CTAs start on items 0 .. grid-1 without asking
+  if (threadIdx.x == 0) {
+    next_item[0] = first_free_item;  // the CTAs start on items 0 .. grid-1 without asking
+    next_item[1] = 0;                // CTAs of the attention kernel that have finished
+  }
   __shared__ int hist[kPlanBuckets];
   for (int i = threadIdx.x; i < kPlanBuckets; i += blockDim.x) hist[i] = 0;
   __syncthreads();
@@ -1028,6 +1031,16 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
   __syncthreads();
   if (tid == 0 && sm.abort_flag != 0) report(a.pool.status, KV_ERR_TIMEOUT);
   if (warp == kWarpProducer) tmem_dealloc(tmem, 512);
+  // The last CTA to finish puts the work counter back where the plan left it, so that the same plan can serve
+  // another launch (a model runs every layer of a step over the same lengths).  a.next_item + 1 counts the CTAs done.
+  if (tid == 0) {
+    __threadfence();
+    if (atomicAdd(a.next_item + 1, 1) == (int)gridDim.x - 1) {
+      a.next_item[0] = (int)gridDim.x;
+      a.next_item[1] = 0;
+      __threadfence();
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1117,14 +1130,16 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                              void* workspace, size_t workspace_bytes, int cta_cap, int mode, const FanArgs* fan,
-                             const AppendArgs* app, cudaStream_t st) {
+                             const AppendArgs* app, int phase, cudaStream_t st) {
+  // phase 0: plan (with the suffix append, if any) and attention; 1: the plan only; 2: attention over the plan that a
+  // phase-1 call with the same arguments left in the workspace
   const size_t need = extend_tc_workspace_bytes(n_q_heads, p->head_dim, batch, total_q, max_total_len);
   if (workspace == nullptr || workspace_bytes < need) return KV_ERR_WORKSPACE;
   const int G = n_q_heads / p->n_kv_heads;
   // Q is read through a tensor map (16-byte base), O is written with 32-byte stores
   if ((reinterpret_cast<uintptr_t>(q) & 15) != 0 || (reinterpret_cast<uintptr_t>(out) & 31) != 0) return KV_ERR_INVALID;
   CUtensorMap q_map;
-  {
+  if (phase != 1) {
     const kv_status_t ms = make_q_map(&q_map, q, total_q, n_q_heads, p->head_dim, G);
     if (ms != KV_OK) return ms;
   }
@@ -1151,7 +1166,9 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   groups = groups > kPlanBuckets / 16 ? kPlanBuckets / 16 : groups;
   const PlanArgs pa{prefix_lens, extend_lens, cu_q, batch, max_tp, lg, max_steps, (int)capacity, max_pages, mode,
                     fan != nullptr ? *fan : FanArgs{}, groups, p->d_status, items, n_items, n_items + 1, grid};
-  if (app != nullptr && app->total_new > 0) {
+  if (phase == 2) {
+    // the plan is in the workspace already
+  } else if (app != nullptr && app->total_new > 0) {
     // plan block + append blocks (32 warps each, one warp per token, all blocks resident at once)
     const int64_t want = ((int64_t)app->total_new + 31) / 32;
     const int64_t cap = 2 * (int64_t)sm_count_of(p->device) - 1;
@@ -1160,8 +1177,11 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   } else {
     extend_tc_plan_kernel<<<1, 1024, 0, st>>>(pa);
   }
-  count_launch();
-  KV_CUDA_OK(cudaGetLastError());
+  if (phase != 2) {
+    count_launch();
+    KV_CUDA_OK(cudaGetLastError());
+  }
+  if (phase == 1) return KV_OK;
 
   TcArgs a{};
   a.pool = p->view();

@@ -23,7 +23,7 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
                              int max_pages, const int* prefix_lens, const int* extend_lens, int batch, int total_q,
                              int max_extend_len, int max_total_len, float scale, void* out, float* lse,
                              void* workspace, size_t workspace_bytes, int cta_cap, int mode, const FanArgs* fan,
-                             const AppendArgs* app, cudaStream_t st);
+                             const AppendArgs* app, int phase, cudaStream_t st);
 kv_status_t launch_extend_small(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                                 int max_pages, const int* prefix_lens, const int* extend_lens, int batch,
                                 int max_extend_len, int max_total_len, float scale, void* out, float* lse,
@@ -148,7 +148,7 @@ kv_status_t launch_extend_shared(kv_pool_t* p, const void* q, int n_q_heads, con
     FanArgs fan{cu_q, cu_children, child_tables, max_pages_child, n_children};
     return launch_extend_tc(p, q, n_q_heads, cu_q_parent, parent_tables, max_pages_parent, parent_lens, rows_parent,
                             n_parents, total_q, max_parent_rows, max_parent_len + max_parent_rows, scale, out, lse, ws,
-                            tc_bytes, 0, 2, &fan, nullptr, st);
+                            tc_bytes, 0, 2, &fan, nullptr, 0, st);
   }
   // part B first, straight into the caller's buffers: each child's suffix over its private pages
   if (!extend_tc_supported(p, n_q_heads))
@@ -156,12 +156,12 @@ kv_status_t launch_extend_shared(kv_pool_t* p, const void* q, int n_q_heads, con
                             max_child_len, max_child_len, scale, out, lse, st);
   else
     s = launch_extend_tc(p, q, n_q_heads, cu_q, child_tables, max_pages_child, zeros, child_lens, n_children, total_q,
-                         max_child_len, max_child_len, scale, out, lse, ws, tc_bytes, 0, 0, nullptr, nullptr, st);
+                         max_child_len, max_child_len, scale, out, lse, ws, tc_bytes, 0, 0, nullptr, nullptr, 0, st);
   if (s != KV_OK) return s;
   if (max_parent_len <= 0) return KV_OK;
   // part A: the stacked suffix rows of each parent over the parent's prefix pages
   s = launch_extend_tc(p, q, n_q_heads, cu_q_parent, parent_tables, max_pages_parent, parent_lens, rows_parent, n_parents,
-                       total_q, max_parent_rows, max_parent_len, scale, o_a, lse_a, ws, tc_bytes, 0, 1, nullptr, nullptr, st);
+                       total_q, max_parent_rows, max_parent_len, scale, o_a, lse_a, ws, tc_bytes, 0, 1, nullptr, nullptr, 0, st);
   if (s != KV_OK) return s;
   const int64_t total = (int64_t)total_q * n_q_heads;
   const unsigned blocks = (unsigned)((total + 7) / 8);

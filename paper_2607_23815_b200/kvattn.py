@@ -62,6 +62,8 @@ _SIGNATURES = {
     "attn_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I, _I]),
     "attn_extend": (_I, [_P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_extend_append": (_I, [_P, _P, _P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
+    "attn_extend_plan": (_I, [_P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _P, _SZ, _P]),
+    "attn_extend_planned": (_I, [_P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_extend_host_staging_bytes": (_SZ, [_P, _I, _I, _I, _I, _I]),
     "attn_extend_host": (_I, [_P, _P, _P, _P, _I, _P, _P, _I, _P, _P, _I, _I, _I, _I, _F, _P, _P, _P, _SZ, _P]),
     "attn_extend_shared_workspace_bytes": (_SZ, [_P, _I, _I, _I, _I, _I]),
@@ -268,6 +270,25 @@ def attn_extend_append(pool: Pool, q, k_new, v_new, cu_q, block_tables, prefix_l
                                     float(scale), _dev_ptr(out), _dev_ptr(lse), _dev_ptr(workspace),
                                     0 if workspace is None else workspace.numel() * workspace.element_size(),
                                     _stream(stream)), "attn_extend_append")
+
+
+def attn_extend_plan(pool: Pool, n_q_heads, cu_q, block_tables, prefix_lens, extend_lens, total_q, max_extend_len,
+                     max_total_len, workspace, stream=None):
+    """Builds attn_extend's work list for these lengths into the workspace (once per step, reused by every layer)."""
+    _check(lib().attn_extend_plan(pool.handle, n_q_heads, _dev_ptr(cu_q), _dev_ptr(block_tables), block_tables.shape[1],
+                                  _dev_ptr(prefix_lens), _dev_ptr(extend_lens), prefix_lens.numel(), total_q,
+                                  max_extend_len, max_total_len, _dev_ptr(workspace),
+                                  workspace.numel() * workspace.element_size(), _stream(stream)), "attn_extend_plan")
+
+
+def attn_extend_planned(pool: Pool, q, cu_q, block_tables, prefix_lens, extend_lens, max_extend_len, max_total_len, scale,
+                        out, lse, workspace, stream=None):
+    """attn_extend over the plan that attn_extend_plan left in the workspace (same arguments)."""
+    _check(lib().attn_extend_planned(pool.handle, _dev_ptr(q), q.shape[1], _dev_ptr(cu_q), _dev_ptr(block_tables),
+                                     block_tables.shape[1], _dev_ptr(prefix_lens), _dev_ptr(extend_lens),
+                                     prefix_lens.numel(), q.shape[0], max_extend_len, max_total_len, float(scale),
+                                     _dev_ptr(out), _dev_ptr(lse), _dev_ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream)), "attn_extend_planned")
 
 
 def attn_extend_host_staging_bytes(pool: Pool, n_q_heads, batch, total_q, max_pages, max_total_len) -> int:

@@ -171,6 +171,17 @@ class DeviceWorkload:
         kvattn.attn_extend_append(self.pool, e.q, e.k_new, e.v_new, e.cu_q, e.block_tables, e.prefix_lens, e.extend_lens,
                                   e.max_extend, e.max_total, self.geom.scale, e.out, e.lse, self.workspace, stream)
 
+    def extend_plan(self, stream=None):
+        e = self.ext
+        kvattn.attn_extend_plan(self.pool, self.geom.n_q_heads, e.cu_q, e.block_tables, e.prefix_lens, e.extend_lens,
+                                e.total_q, e.max_extend, e.max_total, self.workspace, stream)
+
+    def extend_planned(self, stream=None):
+        """attn_extend over the plan extend_plan() left in the workspace (what every layer after the first would call)."""
+        e = self.ext
+        kvattn.attn_extend_planned(self.pool, e.q, e.cu_q, e.block_tables, e.prefix_lens, e.extend_lens, e.max_extend,
+                                   e.max_total, self.geom.scale, e.out, e.lse, self.workspace, stream)
+
     def decode(self, stream=None):
         d = self.dec
         kvattn.attn_decode(self.pool, d.q, d.block_tables, d.ctx_lens, d.max_ctx, self.geom.scale, d.out, d.lse,

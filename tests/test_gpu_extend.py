@@ -284,3 +284,40 @@ def test_append_and_extend_in_one_call_is_bit_identical_to_the_two_calls(impl, h
     assert np.array_equal(imgs[0][0], imgs[1][0]) and np.array_equal(imgs[0][1], imgs[1][1])   # K and V pool images
     assert np.array_equal(outs[0]["o_bits"], outs[1]["o_bits"])
     assert np.array_equal(outs[0]["lse_raw"], outs[1]["lse_raw"])
+
+
+@pytest.mark.parametrize("impl", IMPLS)
+def test_one_plan_serves_several_attention_calls(impl):
+    # attn_extend_plan once, attn_extend_planned several times (a model's layers share the lengths): each call gives
+    # the bits of attn_extend, also when the queries change between the calls.
+    geom = synth.Geometry(32, 8, 128)
+    _skip_if_no_tc(impl, geom)
+    P, E = [0, 300, 17, 1200, 64], [129, 40, 300, 7, 64]
+    L = [p + e for p, e in zip(P, E)]
+    dp = DualPool(geom, 200, seed=555)
+    b = Batch(dp, L)
+    b.write([(i, 0, L[i]) for i in range(len(P))])
+    ref = run_extend(dp, b, P, E, impl=impl)
+    assert_close(ref, "plain call")
+    t = lambda x: torch.tensor(np.asarray(x), dtype=torch.int32, device="cuda")
+    cu, bt, pl, el = t(np.concatenate([[0], np.cumsum(E)])), torch.from_numpy(b.block_tables()).to("cuda"), t(P), t(E)
+    q = ref["q"]
+    ws = torch.empty(kvattn.attn_workspace_bytes(dp.pool, 32, len(P), int(q.shape[0]), max(L), 0, 0), dtype=torch.uint8,
+                     device="cuda")
+    kvattn.kvattn_set_extend_impl(impl)
+    try:
+        kvattn.attn_extend_plan(dp.pool, 32, cu, bt, pl, el, int(q.shape[0]), max(E), max(L), ws)
+        for rep in range(4):
+            qq = q if rep != 2 else (-q).contiguous()                # another layer's queries over the same plan
+            out = torch.full_like(q, float("nan"))
+            lse = torch.full((q.shape[0], 32), float("nan"), dtype=torch.float32, device="cuda")
+            kvattn.attn_extend_planned(dp.pool, qq, cu, bt, pl, el, max(E), max(L), geom.scale, out, lse, ws)
+            torch.cuda.synchronize()
+            if rep != 2:
+                assert np.array_equal(synth.bf16_bits(out), ref["o_bits"]) and np.array_equal(lse.cpu().numpy(), ref["lse_raw"])
+            else:
+                assert torch.isfinite(out.float()).all() and not np.array_equal(synth.bf16_bits(out), ref["o_bits"])
+    finally:
+        kvattn.kvattn_set_extend_impl(0)
+    assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+    dp.close()
