@@ -292,9 +292,9 @@ typedef struct {
  * extend set and the decode set are launched so that the tensor-bound and the HBM-bound work
  * share the GPU.  Either argument may be NULL or have batch 0.  The workspace must be sized by
  * attn_workspace_bytes() with both batches.  Work is ordered after prior work on `stream`, and
- * later work on `stream` is ordered after it.  The call uses a side stream and a pair of events that
- * belong to the pool: two attn_mixed calls on the same pool must not be issued concurrently from two
- * threads, nor on two different caller streams without an ordering between them. */
+ * later work on `stream` is ordered after it: both kernels are queued on `stream` itself, the decode kernel so that
+ * it starts beside the extend kernel instead of behind it.  The extend kernel takes a share of the SMs that is
+ * derived from the host-side bounds of the two batches (kvattn_set_mixed_extend_ctas overrides it). */
 kv_status_t attn_mixed(kv_pool_t* pool, int n_q_heads, float scale, const attn_extend_args_t* ext,
                        const attn_decode_args_t* dec, void* workspace, size_t workspace_bytes, void* stream);
 
@@ -313,8 +313,13 @@ kv_status_t kvattn_set_extend_impl(int impl);
 /* Test/tuning hook for attn_extend_shared: 0 = choose by the mean suffix length (default), 1 = three kernels
  * (shared part, own part, merge), 2 = one kernel that walks the parent's and then the children's tiles. */
 kv_status_t kvattn_set_shared_impl(int impl);
+/* Selects how the decode kernel brings pages on chip: 0 = default, 1 = straight into registers (one page per warp in
+ * flight), 2 = through a per-warp ring of page slots in shared memory filled by bulk copies (several pages per warp in
+ * flight).  Same arithmetic, same bits.  Process-wide; for tests and benchmarks. */
+kv_status_t kvattn_set_decode_impl(int impl);
 /* Tuning: inside attn_mixed (both sets present) the persistent extend kernel takes at most n SMs, so that the
- * HBM-bound decode kernel runs beside it on the others instead of after it.  0 = no limit.  Process-wide. */
+ * HBM-bound decode kernel runs beside it on the others instead of after it.  0 = derived from the bounds of the two
+ * batches (the default).  Process-wide. */
 kv_status_t kvattn_set_mixed_extend_ctas(int n);
 /* Test surface (the paper has no counterpart): runs a one-CTA kernel whose warps wait, with the same bounded
  * wait the attention kernels use, on barriers that nothing completes; the first gives up after limit_ns

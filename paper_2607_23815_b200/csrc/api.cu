@@ -6,7 +6,7 @@ namespace kvattn {
 size_t decode_workspace_bytes(int n_q_heads, int head_dim, int batch, int max_ctx_len);
 kv_status_t launch_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
                           const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
-                          void* workspace, size_t workspace_bytes, cudaStream_t st);
+                          void* workspace, size_t workspace_bytes, cudaStream_t st, bool beside = false);
 kv_status_t launch_extend_small(kv_pool_t* p, const void* q, int n_q_heads, const int* cu_q, const int* block_tables,
                                 int max_pages, const int* prefix_lens, const int* extend_lens, int batch,
                                 int max_extend_len, int max_total_len, float scale, void* out, float* lse,
@@ -29,6 +29,7 @@ kv_status_t launch_extend_shared(kv_pool_t* p, const void* q, int n_q_heads, con
                                  cudaStream_t st);
 
 extern std::atomic<int> g_shared_impl;
+extern std::atomic<int> g_decode_impl;
 
 static std::atomic<int> g_extend_impl{0};
 static std::atomic<int> g_mixed_extend_ctas{0};  // SMs the extend kernel may take inside attn_mixed (0 = all)
@@ -270,15 +271,21 @@ kv_status_t kvattn_set_shared_impl(int impl) {
   return KV_OK;
 }
 
+kv_status_t kvattn_set_decode_impl(int impl) {
+  if (impl < 0 || impl > 2) return KV_ERR_INVALID;
+  g_decode_impl.store(impl);
+  return KV_OK;
+}
+
 kv_status_t kvattn_set_mixed_extend_ctas(int n) {
   if (n < 0) return KV_ERR_INVALID;
   g_mixed_extend_ctas.store(n);
   return KV_OK;
 }
 
-kv_status_t attn_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
-                        const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
-                        void* workspace, size_t workspace_bytes, void* stream) {
+static kv_status_t decode_impl(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
+                               const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
+                               void* workspace, size_t workspace_bytes, void* stream, bool beside) {
   if (p == nullptr || batch < 0 || max_pages < 0 || max_ctx_len < 0) return KV_ERR_INVALID;
   if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
   if (batch == 0) return KV_OK;
@@ -291,7 +298,14 @@ kv_status_t attn_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* b
   // the decode region of a combined workspace starts after the extend region; a caller that sized
   // the workspace for decode only passes (0, 0) for the extend part, so the offset is 0 there
   return launch_decode(p, q, n_q_heads, block_tables, max_pages, ctx_lens, batch, max_ctx_len, scale, out, lse,
-                       workspace, workspace_bytes, (cudaStream_t)stream);
+                       workspace, workspace_bytes, (cudaStream_t)stream, beside);
+}
+
+kv_status_t attn_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
+                        const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
+                        void* workspace, size_t workspace_bytes, void* stream) {
+  return decode_impl(p, q, n_q_heads, block_tables, max_pages, ctx_lens, batch, max_ctx_len, scale, out, lse, workspace,
+                     workspace_bytes, stream, false);
 }
 
 kv_status_t attn_mixed(kv_pool_t* p, int n_q_heads, float scale, const attn_extend_args_t* ext,
@@ -307,22 +321,27 @@ kv_status_t attn_mixed(kv_pool_t* p, int n_q_heads, float scale, const attn_exte
   if (ext_bytes > workspace_bytes) return KV_ERR_WORKSPACE;
   char* ws = reinterpret_cast<char*>(workspace);
   if (has_ext && has_dec) {
-    // The persistent extend kernel (tensor-bound) goes first on the caller's stream and may be limited to a
-    // part of the SMs; decode (HBM-bound) follows on the pool's side stream and fills the others.
-    KV_CUDA_OK(cudaEventRecord(p->ev_fork, st));
-    KV_CUDA_OK(cudaStreamWaitEvent(p->side_stream, p->ev_fork, 0));
+    // Both kernels go to the caller's stream.  The persistent extend kernel (tensor-bound) is limited to a share of
+    // the SMs and lets the kernel queued behind it start as soon as its own CTAs are resident; the decode kernel
+    // (HBM-bound) is queued with the early-start attribute, fills the other SMs at once and, block after block, the
+    // SMs the extend CTAs give back.  It waits for nothing: it reads and writes nothing the extend kernel writes.
+    int cap = g_mixed_extend_ctas.load();
+    if (cap <= 0) {
+      // Share of the SMs by the two kinds of work, from the host-side bounds: extend costs its flops at the rate the
+      // kernel reaches per SM, decode its bytes at the rate at which about two thirds of the SMs saturate the memory.
+      const int sms = sm_count_of(p->device);
+      const double flops = 4.0 * p->head_dim * n_q_heads * (double)ext->total_q * 0.75 * ext->max_total_len;
+      const double bytes = (double)dec->batch * 0.62 * dec->max_ctx_len * 2.0 * p->n_kv_heads * p->head_dim * 2.0;
+      const double sm_s_ext = flops / 800e12 * sms, sm_s_dec = bytes / 6e12 * (sms * 0.68);
+      cap = (int)(sms * sm_s_ext / (sm_s_ext + sm_s_dec) + 0.5);
+      cap = cap < 16 ? 16 : (cap > sms - 32 ? sms - 32 : cap);
+    }
     kv_status_t s = extend_impl(p, ext->q, n_q_heads, ext->cu_q, ext->block_tables, ext->max_pages, ext->prefix_lens,
                                 ext->extend_lens, ext->batch, ext->total_q, ext->max_extend_len, ext->max_total_len,
-                                scale, ext->out, ext->lse, ws, ext_bytes, g_mixed_extend_ctas.load() > 0 ? g_mixed_extend_ctas.load() : -1, st);
-    kv_status_t s2 = KV_OK;
-    if (s == KV_OK)
-      s2 = attn_decode(p, dec->q, n_q_heads, dec->block_tables, dec->max_pages, dec->ctx_lens, dec->batch,
-                       dec->max_ctx_len, scale, dec->out, dec->lse, ws ? ws + ext_bytes : nullptr,
-                       workspace_bytes - ext_bytes, p->side_stream);
-    // always rejoin, so that the caller's stream stays ordered after whatever was launched
-    KV_CUDA_OK(cudaEventRecord(p->ev_join, p->side_stream));
-    KV_CUDA_OK(cudaStreamWaitEvent(st, p->ev_join, 0));
-    return s != KV_OK ? s : s2;
+                                scale, ext->out, ext->lse, ws, ext_bytes, cap, st);
+    if (s != KV_OK) return s;
+    return decode_impl(p, dec->q, n_q_heads, dec->block_tables, dec->max_pages, dec->ctx_lens, dec->batch, dec->max_ctx_len,
+                       scale, dec->out, dec->lse, ws ? ws + ext_bytes : nullptr, workspace_bytes - ext_bytes, st, true);
   }
   if (has_ext)
     return attn_extend(p, ext->q, n_q_heads, ext->cu_q, ext->block_tables, ext->max_pages, ext->prefix_lens,

@@ -12,7 +12,7 @@ namespace kvattn {
 size_t decode_workspace_bytes(int n_q_heads, int head_dim, int batch, int max_ctx_len);
 kv_status_t launch_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
                           const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
-                          void* workspace, size_t workspace_bytes, cudaStream_t st);
+                          void* workspace, size_t workspace_bytes, cudaStream_t st, bool beside = false);
 
 constexpr size_t kStaticScratchBytes = size_t(8) << 20;  // 8 MiB, held by every GPU that loads the library
 

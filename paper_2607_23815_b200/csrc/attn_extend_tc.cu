@@ -438,6 +438,9 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
     if (threadIdx.x == 0) report(a.pool.status, KV_ERR_CUDA);
     return;
   }
+  // A kernel queued behind this one with the early-start attribute may take the SMs this grid leaves free as soon as
+  // every CTA of this grid is resident (the mixed step queues the decode kernel that way).
+  launch_dependents();
   TcSmem<D>& sm = *reinterpret_cast<TcSmem<D>*>(smem_raw);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   volatile int* abortp = &sm.abort_flag;

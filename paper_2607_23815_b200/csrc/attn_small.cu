@@ -10,6 +10,7 @@
 // maximum is shared with three shuffles per page, the row sum is reduced once at the end.
 // Partial results of the chunks are merged by combine_kernel with the log-sum-exp rule.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace kvattn {
 
@@ -97,13 +98,78 @@ __device__ __forceinline__ void load_page(PageRegs<D>& pr, const char* kblk, con
   }
 }
 
-template <int D, bool EXTEND, bool DIRECT>
-__global__ void __launch_bounds__(256, 1) attn_small_kernel(SmallArgs a, int64_t total_items) {
+// ---- ring variant (decode): pages come through shared memory -----------------------------------------------
+// The register-streaming loader above keeps one page per warp in flight, which is what the registers allow; a warp
+// then waits out most of every page's latency, and only all SMs together reach the memory's bandwidth.  In the ring
+// variant every warp owns kRingStages page slots in shared memory that it fills with bulk copies (one 16-token K block
+// and one V block per slot, exactly as they lie in the pool), so kRingStages - 1 pages per warp are in flight while one
+// is consumed, whatever the register budget: fewer SMs saturate HBM, which leaves the others to the tensor-core
+// kernel in a mixed step.  The arithmetic on a page is the same code, so the results are the same bits.
+constexpr int kRingWarps = 8;
+constexpr int kRingStages = 3;
+
+template <int D>
+constexpr int ring_smem_bytes() { return kRingWarps * kRingStages * 2 * 16 * D * 2 + kRingWarps * kRingStages * 8 + 16; }
+
+// Fragments of one page from a shared-memory slot (K block, then V block).  Within a quarter warp the K loads of the
+// lanes with an odd row take the other 64-byte half first (j ^ 1), so that the eight lanes touch eight different
+// 16-byte bank groups; the registers are swapped back afterwards.
+template <int D>
+__device__ __forceinline__ void load_page_smem(PageRegs<D>& pr, uint32_t slot, int r, int c) {
+  auto lds = [](uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+  };
+  const int flip = r & 1;
+#pragma unroll
+  for (int g = 0; g < 2; ++g) {
+#pragma unroll
+    for (int j = 0; j < D / 32; ++j) {
+      const int ch = 4 * (j ^ flip) + c;
+      pr.k[g][j] = lds(slot + g * (D * 16) + (ch >> 3) * 1024 + r * 128 + (((ch & 7) ^ r) << 4));
+    }
+    if (flip) {
+#pragma unroll
+      for (int j = 0; j < D / 32; j += 2) {
+        const uint4 t = pr.k[g][j];
+        pr.k[g][j] = pr.k[g][j + 1];
+        pr.k[g][j + 1] = t;
+      }
+    }
+  }
+  const uint32_t vslot = slot + 16 * D * 2;
+#pragma unroll
+  for (int g = 0; g < 2; ++g) {
+#pragma unroll
+    for (int par = 0; par < 2; ++par) {
+      const int row = 2 * c + par;
+#pragma unroll
+      for (int u = 0; u < D / 64; ++u)
+        pr.v[g][par][u] = lds(vslot + g * (D * 16) + u * 1024 + row * 128 + ((r ^ row) << 4));
+    }
+  }
+}
+
+template <int D, bool EXTEND, bool DIRECT, bool RING = false>
+__global__ void __launch_bounds__(RING ? kRingWarps * 32 : 256, 1) attn_small_kernel(SmallArgs a, int64_t total_items) {
+  constexpr int kWarps = RING ? kRingWarps : 8;
+  constexpr int kBatchPages = RING ? 2 * kChunkPages : kChunkPages;  // block-table entries held per lane pair / lane
+  extern __shared__ __align__(1024) unsigned char ring_raw[];
+  unsigned long long* ring_bars = reinterpret_cast<unsigned long long*>(ring_raw + kRingWarps * kRingStages * 2 * 16 * D * 2);
+  int* ring_abort = reinterpret_cast<int*>(ring_bars + kRingWarps * kRingStages);
+  if (RING) {
+    if (threadIdx.x == 0) *ring_abort = 0;
+    if ((threadIdx.x & 31) == 0)
+      for (int s = 0; s < kRingStages; ++s) ptx::mbar_init(ptx::smem_u32(&ring_bars[(threadIdx.x >> 5) * kRingStages + s]), 1);
+    ptx::fence_mbar_init();
+    __syncthreads();
+  }
   constexpr int NJ = D / 32;  // K chunk loads per token row per lane
   constexpr int NU = D / 64;  // 64-dim halves
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int r = lane >> 2, c = lane & 3;
-  const int64_t item = (int64_t)blockIdx.x * 8 + warp;
+  const int64_t item = (int64_t)blockIdx.x * kWarps + warp;
   if (item >= total_items) return;
 
   const int Hkv = a.pool.n_kv_heads, G = a.group, Hq = a.n_q_heads;
@@ -188,17 +254,24 @@ __global__ void __launch_bounds__(256, 1) attn_small_kernel(SmallArgs a, int64_t
   const int first_page = chunk_begin >> 4;
   const int n_pages = (chunk_end - chunk_begin + 15) >> 4;
 
-  for (int pb = 0; pb < n_pages; pb += kChunkPages) {
-    const int np = min(kChunkPages, n_pages - pb);
-    int my_page = 0;
-    if (lane < np) {
-      const int b = first_page + pb + lane;
-      my_page = (b < a.max_pages) ? __ldg(bt_row + b) : -1;
-      if ((unsigned)my_page >= (unsigned)a.pool.num_pages) {
-        report(a.pool.status, KV_ERR_BOUNDS);
-        my_page = 0;  // stay inside the pool; the result of this row is flagged, not trusted
+  uint32_t ring_issued = 0, ring_used = 0;  // ring variant: pages asked for / consumed so far (slot and phase follow)
+  for (int pb = 0; pb < n_pages; pb += kBatchPages) {
+    const int np = min(kBatchPages, n_pages - pb);
+    int my_page = 0, my_page_hi = 0;
+    auto table_entry = [&](int idx) {
+      int pg = 0;
+      if (idx < np) {
+        const int b = first_page + pb + idx;
+        pg = (b < a.max_pages) ? __ldg(bt_row + b) : -1;
+        if ((unsigned)pg >= (unsigned)a.pool.num_pages) {
+          report(a.pool.status, KV_ERR_BOUNDS);
+          pg = 0;  // stay inside the pool; the result of this row is flagged, not trusted
+        }
       }
-    }
+      return pg;
+    };
+    my_page = table_entry(lane);
+    if (RING) my_page_hi = table_entry(lane + 32);
     // one page of work on the registers in `pr`
     auto process = [&](PageRegs<D>& pr, int p) {
       const int tok0 = chunk_begin + ((pb + p) << 4);  // first token of this page
@@ -274,15 +347,58 @@ __global__ void __launch_bounds__(256, 1) attn_small_kernel(SmallArgs a, int64_t
       load_page<D>(pr, kbase + (size_t)pg * page_stride, vbase + (size_t)pg * page_stride, r, c);
     };
 
-    // two register sets alternate: the next page's loads are in flight while this one is consumed
-    PageRegs<D> ra, rb;
-    fetch(ra, 0);
-    for (int p = 0; p < np; p += 2) {
-      if (p + 1 < np) fetch(rb, p + 1);
-      process(ra, p);
-      if (p + 1 < np) {
-        if (p + 2 < np) fetch(ra, p + 2);
-        process(rb, p + 1);
+    if constexpr (RING) {
+      const uint32_t slots = ptx::smem_u32(ring_raw) + warp * (kRingStages * 2 * 16 * D * 2);
+      const uint32_t bars = ptx::smem_u32(&ring_bars[warp * kRingStages]);
+      // asks for page p of the batch into the next slot of the ring (whole warp calls; lane 0 issues)
+      auto issue = [&](int p) {
+        const int pg = p < 32 ? __shfl_sync(0xffffffffu, my_page, p & 31) : __shfl_sync(0xffffffffu, my_page_hi, p & 31);
+        if (lane == 0) {
+          const uint32_t s = ring_issued % kRingStages;
+          const uint32_t slot = slots + s * (2 * 16 * D * 2), bar = bars + s * 8;
+          ptx::mbar_arrive_expect_tx(bar, 2 * 16 * D * 2);
+          ptx::bulk_g2s(slot, kbase + (size_t)pg * page_stride, 16 * D * 2, bar);
+          ptx::bulk_g2s(slot + 16 * D * 2, vbase + (size_t)pg * page_stride, 16 * D * 2, bar);
+        }
+        ++ring_issued;
+      };
+      for (int p = 0; p < min(kRingStages, np); ++p) issue(p);
+      PageRegs<D> pr;
+      bool ok = true;
+      for (int p = 0; p < np && ok; ++p) {
+        const uint32_t s = ring_used % kRingStages;
+        ok = ptx::mbar_wait(bars + s * 8, (ring_used / kRingStages) & 1, ring_abort);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        ++ring_used;
+        load_page_smem<D>(pr, slots + s * (2 * 16 * D * 2), r, c);
+        // every lane has its copy of the slot in registers: the slot can take the page kRingStages ahead
+        __syncwarp();
+        ptx::fence_proxy_async_smem();
+        if (p + kRingStages < np) issue(p + kRingStages);
+        process(pr, p);
+      }
+      if (!ok) {
+        // a wait gave up: flag it, let the copies that were asked for land (bounded), and leave
+        if (lane == 0) {
+          report(a.pool.status, KV_ERR_TIMEOUT);
+          int never = 0;
+          for (; ring_used < ring_issued; ++ring_used)
+            ptx::mbar_wait_limit(bars + (ring_used % kRingStages) * 8, (ring_used / kRingStages) & 1, &never, 100000000ull);
+        }
+        return;
+      }
+    } else {
+      // two register sets alternate: the next page's loads are in flight while this one is consumed
+      PageRegs<D> ra, rb;
+      fetch(ra, 0);
+      for (int p = 0; p < np; p += 2) {
+        if (p + 1 < np) fetch(rb, p + 1);
+        process(ra, p);
+        if (p + 1 < np) {
+          if (p + 2 < np) fetch(ra, p + 2);
+          process(rb, p + 1);
+        }
       }
     }
   }
@@ -384,18 +500,70 @@ size_t decode_workspace_bytes(int n_q_heads, int head_dim, int batch, int max_ct
   return align256(slots * head_dim * sizeof(float)) + align256(slots * sizeof(float));
 }
 
+std::atomic<int> g_decode_impl{0};  // 0: default, 1: pages stream through registers, 2: pages go through a shared-memory ring
+
+// Launches the partial (or direct) decode kernel in the chosen variant.
+template <int D, bool DIRECT>
+// beside: the kernel is launched so that it may start while the kernel in front of it in the stream still runs (it does
+// not wait for it: nothing it touches is written there).  The mixed step uses this to run decode next to the extend kernel.
+static kv_status_t launch_decode_kernel(kv_pool_t* p, const SmallArgs& a, int64_t items, bool ring, bool beside, cudaStream_t st) {
+  cudaLaunchConfig_t cfg{};
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = beside ? 1 : 0;
+  if (ring) {
+    constexpr int smem = ring_smem_bytes<D>();
+    static std::atomic<bool> configured[kMaxDevices];
+    if (p->device < 0 || p->device >= kMaxDevices) return KV_ERR_INVALID;
+    if (!configured[p->device].load(std::memory_order_acquire)) {
+      KV_CUDA_OK(cudaFuncSetAttribute(attn_small_kernel<D, false, DIRECT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+      configured[p->device].store(true, std::memory_order_release);
+    }
+    cfg.gridDim = dim3((unsigned)((items + kRingWarps - 1) / kRingWarps));
+    cfg.blockDim = dim3(kRingWarps * 32);
+    cfg.dynamicSmemBytes = smem;
+    KV_CUDA_OK(cudaLaunchKernelEx(&cfg, attn_small_kernel<D, false, DIRECT, true>, a, items));
+  } else {
+    cfg.gridDim = dim3((unsigned)((items + 7) / 8));
+    cfg.blockDim = dim3(256);
+    KV_CUDA_OK(cudaLaunchKernelEx(&cfg, attn_small_kernel<D, false, DIRECT, false>, a, items));
+  }
+  return KV_OK;
+}
+
 template <int D>
 static kv_status_t launch_decode_d(kv_pool_t* p, const SmallArgs& base, int batch, int max_ctx_len, void* workspace,
-                                   size_t workspace_bytes, cudaStream_t st) {
+                                   size_t workspace_bytes, bool beside, cudaStream_t st) {
   SmallArgs a = base;
+  // beside the tensor-core kernel the ring variant is the default: it keeps more bytes in flight per SM, so the SMs the
+  // other kernel leaves free come closer to the memory's bandwidth (measured: mixed step 0.46 -> 0.42 ms)
+  const int impl = g_decode_impl.load();
+  const bool ring = impl == 2 || (impl == 0 && beside);
   a.max_row_tiles = 1;
   a.chunk_tokens = kDecodeChunkTokens;
   a.max_chunks = (max_ctx_len + kDecodeChunkTokens - 1) / kDecodeChunkTokens;
   const int64_t items = (int64_t)batch * p->n_kv_heads * a.max_chunks;
-  const int blocks = (int)((items + 7) / 8);
   if (a.max_chunks == 1) {
-    fill_empty_rows_kernel<<<batch, 128, 0, st>>>(a.len_a, batch, a.n_q_heads * D, a.out, a.lse, a.n_q_heads);
-    attn_small_kernel<D, false, true><<<blocks, 256, 0, st>>>(a, items);
+    // (the two kernels write disjoint rows: the second need not wait for the first either)
+    if (beside) {
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3((unsigned)batch);
+      cfg.blockDim = dim3(128);
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      KV_CUDA_OK(cudaLaunchKernelEx(&cfg, fill_empty_rows_kernel, a.len_a, batch, a.n_q_heads * D, a.out, a.lse, a.n_q_heads));
+    } else {
+      fill_empty_rows_kernel<<<batch, 128, 0, st>>>(a.len_a, batch, a.n_q_heads * D, a.out, a.lse, a.n_q_heads);
+    }
+    const kv_status_t ks = launch_decode_kernel<D, true>(p, a, items, ring, beside, st);
+    if (ks != KV_OK) return ks;
     count_launch(2);
   } else {
     const size_t need = decode_workspace_bytes(a.n_q_heads, D, batch, max_ctx_len);
@@ -403,7 +571,8 @@ static kv_status_t launch_decode_d(kv_pool_t* p, const SmallArgs& base, int batc
     const size_t slots = (size_t)batch * a.n_q_heads * a.max_chunks;
     a.part_o = reinterpret_cast<float*>(workspace);
     a.part_lse = reinterpret_cast<float*>(reinterpret_cast<char*>(workspace) + align256(slots * D * sizeof(float)));
-    attn_small_kernel<D, false, false><<<blocks, 256, 0, st>>>(a, items);
+    const kv_status_t ks = launch_decode_kernel<D, false>(p, a, items, ring, beside, st);
+    if (ks != KV_OK) return ks;
     const int rows = batch * a.n_q_heads;
     combine_kernel<D><<<(rows + 7) / 8, 256, 0, st>>>(a.part_o, a.part_lse, a.len_a, batch, a.n_q_heads, a.max_chunks,
                                                       a.chunk_tokens, a.out, a.lse);
@@ -415,7 +584,7 @@ static kv_status_t launch_decode_d(kv_pool_t* p, const SmallArgs& base, int batc
 
 kv_status_t launch_decode(kv_pool_t* p, const void* q, int n_q_heads, const int* block_tables, int max_pages,
                           const int* ctx_lens, int batch, int max_ctx_len, float scale, void* out, float* lse,
-                          void* workspace, size_t workspace_bytes, cudaStream_t st) {
+                          void* workspace, size_t workspace_bytes, cudaStream_t st, bool beside) {
   SmallArgs a{};
   a.pool = p->view();
   a.q = (const __nv_bfloat16*)q;
@@ -428,8 +597,8 @@ kv_status_t launch_decode(kv_pool_t* p, const void* q, int n_q_heads, const int*
   a.scale_log2 = scale * 1.4426950408889634f;
   a.out = (__nv_bfloat16*)out;
   a.lse = lse;
-  if (p->head_dim == 128) return launch_decode_d<128>(p, a, batch, max_ctx_len, workspace, workspace_bytes, st);
-  return launch_decode_d<64>(p, a, batch, max_ctx_len, workspace, workspace_bytes, st);
+  if (p->head_dim == 128) return launch_decode_d<128>(p, a, batch, max_ctx_len, workspace, workspace_bytes, beside, st);
+  return launch_decode_d<64>(p, a, batch, max_ctx_len, workspace, workspace_bytes, beside, st);
 }
 
 // Extend on the small-tile kernel: every tile of 8 query rows walks its whole visible KV range

@@ -78,9 +78,6 @@ struct kv_pool {
   uint64_t clock;
   uint32_t mark_epoch;
   int64_t evicted_total;
-  // second stream + events used by attn_mixed to overlap the two kinds of work
-  cudaStream_t side_stream;
-  cudaEvent_t ev_fork, ev_join;
   // attn_extend_host: copies in and out run on streams of their own, so that they overlap the kernels of the
   // neighbouring steps; per staging area (up to kHostSlots in rotation) the events that order its reuse
   static constexpr int kHostSlots = 4;

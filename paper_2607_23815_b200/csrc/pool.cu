@@ -126,7 +126,6 @@ static kv_status_t pool_create_impl(int num_pages, int page_size, int n_kv_heads
   p->owns_buffers = owns; p->k_base = k_base; p->v_base = v_base;
   p->bytes_each = (int64_t)num_pages * n_kv_heads * (int64_t)block_bytes(head_dim);
   p->d_status = nullptr; p->d_scratch_ids = nullptr; p->poison = false;
-  p->side_stream = nullptr; p->ev_fork = nullptr; p->ev_join = nullptr;
   p->h2d_stream = nullptr; p->d2h_stream = nullptr; p->host_slot_next = 0;
   for (auto& hs : p->host_slots) hs = kv_pool::HostSlot{nullptr, nullptr, nullptr, nullptr};
   p->mark_epoch = 0; p->evicted_total = 0;
@@ -138,9 +137,6 @@ static kv_status_t pool_create_impl(int num_pages, int page_size, int n_kv_heads
   ok = ok && cudaMalloc(&p->d_status, sizeof(int)) == cudaSuccess &&
        cudaMemset(p->d_status, 0, sizeof(int)) == cudaSuccess &&
        cudaMalloc(&p->d_scratch_ids, sizeof(int) * (size_t)num_pages) == cudaSuccess &&
-       cudaStreamCreateWithFlags(&p->side_stream, cudaStreamNonBlocking) == cudaSuccess &&
-       cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) == cudaSuccess &&
-       cudaEventCreateWithFlags(&p->ev_join, cudaEventDisableTiming) == cudaSuccess &&
        cudaStreamCreateWithFlags(&p->h2d_stream, cudaStreamNonBlocking) == cudaSuccess &&
        cudaStreamCreateWithFlags(&p->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
   for (auto& hs : p->host_slots)
@@ -183,9 +179,6 @@ kv_status_t kv_pool_destroy(kv_pool_t* p) {
   }
   if (p->d_status) cudaFree(p->d_status);
   if (p->d_scratch_ids) cudaFree(p->d_scratch_ids);
-  if (p->side_stream) cudaStreamDestroy(p->side_stream);
-  if (p->ev_fork) cudaEventDestroy(p->ev_fork);
-  if (p->ev_join) cudaEventDestroy(p->ev_join);
   if (p->h2d_stream) cudaStreamDestroy(p->h2d_stream);
   if (p->d2h_stream) cudaStreamDestroy(p->d2h_stream);
   for (auto& hs : p->host_slots) {

@@ -77,6 +77,7 @@ _SIGNATURES = {
     "kv_last_async_status": (_I, [_P]),
     "kvattn_set_extend_impl": (_I, [_I]),
     "kvattn_set_shared_impl": (_I, [_I]),
+    "kvattn_set_decode_impl": (_I, [_I]),
     "kvattn_set_mixed_extend_ctas": (_I, [_I]),
     "kvattn_selftest_bounded_wait": (_I, [_P, C.c_ulonglong, _P, _P]),
     "kvattn_launch_count": (_I64, []),
@@ -383,6 +384,10 @@ def kv_last_async_status(pool: Pool) -> int:
 
 def kvattn_set_extend_impl(impl: int):
     _check(lib().kvattn_set_extend_impl(impl), "kvattn_set_extend_impl")
+
+
+def kvattn_set_decode_impl(impl: int):
+    _check(lib().kvattn_set_decode_impl(impl), "kvattn_set_decode_impl")
 
 
 def kvattn_set_mixed_extend_ctas(n: int):
