@@ -7,24 +7,24 @@ and the benchmark's CPU-baseline leg do).
 
 What it computes, and the passages it restates:
 
-* The KV cache is a global pool of fixed-size blocks ("pages"); a request's
-  logical blocks map to physical pages through a block table, pages are handed
-  out on admission and returned on completion (paper Section 2.1, "vLLM memory
+* The KV cache is one pool of equally sized blocks (pages) for all requests; a
+  request's logical blocks map to physical pages through a block table, pages
+  are handed out on admission and given back on completion (paper Section 2.1, "vLLM memory
   model").  -> ``FreeList``, ``PagePool``, ``append``, ``gather``.
 * Prefill materialises K/V for all prompt tokens; decode attends one new token
   over all stored K/V (Section 2.1, first paragraph).  -> ``attn_decode``.
 * With prefix caching the engine reuses the cached KV entries of a shared
   prompt prefix and computes only the novel suffix (Section 2.1, "Prefix
   caching"; Section 2.1, "Prefix sharing in semantic operators": the map
-  operator "only prefills the map-specific suffix").  -> ``attn_extend``.
+  operator prefills nothing but its own suffix).  -> ``attn_extend``.
   The suffix token t of a prompt [S | C(t) | I] sits at absolute position
   P + t, sees every prefix key and the suffix keys up to itself.
 * A Cartesian product turns one finished task into several dependent tasks
   that all reuse the parent's prefix (Section 5.1, "dependent tasks";
   Section 5.3, the Complete procedure).  -> ``attn_extend_shared``: child c of
   parent g sees the parent's P_g keys followed by its own suffix so far.
-* Reuse does not change results (Section 1: scheduling "does not change query
-  semantics or output accuracy").  So the result has a plain definition,
+* Reuse does not change results (Section 1: scheduling leaves the query's
+  meaning and the accuracy of its output untouched).  So the result has a plain definition,
   softmax(q K^T * scale) V over the visible keys, and this oracle is that
   definition written out: gather the sequence's pages into contiguous K/V,
   then three separate passes (max, sum of exponentials, weighted sum) in

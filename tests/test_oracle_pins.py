@@ -120,44 +120,39 @@ def test_zero_keys_closed_form(P, E):
 
 
 def test_planted_needle_names_the_key_that_was_read():
-    # One key per (row, head) is made to dominate; V is position-coded, so the output
-    # reveals which (page, slot, kv head) was read.
-    rng = np.random.default_rng(11)
-    Hq, Hkv, D, ps, P, E = 4, 2, 8, 16, 37, 21
+    # One key per (row, head) is made to dominate; V is position-coded, so the output reveals which (page, slot, kv
+    # head) was read.  Key j carries two one-hot codes (j mod 8 and j div 8) of height 8; a query that carries the
+    # codes of its target scores 128 there and at most 64 anywhere else, so every row of every head is decided by a
+    # margin of 64 and every one of them is checked.
+    Hq, Hkv, D, ps, P, E = 4, 2, 16, 16, 37, 21
     G, L = Hq // Hkv, P + E
-    q = _rand_bits(rng, (E, Hq, D))
-    qf = orc.widen(q)
-    k = np.zeros((L, Hkv, D), np.uint16)
+    kf = np.zeros((L, Hkv, D), np.float32)
     v = np.zeros((L, Hkv, D), np.float32)
     for j in range(L):
+        kf[j, :, j % 8] = 8.0
+        kf[j, :, 8 + j // 8] = 8.0
         for g in range(Hkv):
-            v[j, g, 0::2] = j % 64
+            v[j, g, 0::2] = j
             v[j, g, 1::2] = 100 + g
-    needles = {}
-    # each (t, h) gets its own needle position; one K row per (j, kv head) can serve one query
-    # head only, so plant for one head of each group per row and check those.
-    kf = np.zeros((L, Hkv, D), np.float32)
+    qf = np.zeros((E, Hq, D), np.float32)
+    target = {}
     for t in range(E):
-        for g in range(Hkv):
-            h = g * G + (t % G)
-            j = (7 * t + 3 * g) % (P + t + 1)
-            while (j, g) in needles.values():
-                j = (j + 1) % (P + t + 1)
-            needles[(t, h)] = (j, g)
-            kf[j, g] = 64.0 * qf[t, h] / np.dot(qf[t, h], qf[t, h])   # score 64 for its own query
-    k = synth.bf16_bits(torch.from_numpy(kf).to(torch.bfloat16))
-    vb = synth.bf16_bits(torch.from_numpy(v).to(torch.bfloat16))
+        for h in range(Hq):
+            j = [P + t, 0, (7 * t + 5 * h) % (P + t + 1), 16 * ((P + t) // 16)][(t + h) % 4]   # diagonal, first, any, page start
+            target[(t, h)] = j
+            qf[t, h, j % 8] = 8.0
+            qf[t, h, 8 + j // 8] = 8.0
+    bits = lambda x: synth.bf16_bits(torch.from_numpy(x).to(torch.bfloat16))
     pool = orc.PagePool(32, ps, Hkv, D, fill=0x7FC0)
     pages = synth.page_permutation(9, 32).tolist()[:synth.pages_needed(L, ps)]
-    pool.append(pages, 0, k, vb)
-    o, _ = orc.attn_extend(pool, q, Hq, [0, E], synth.block_table([pages]), [P], [E], 1.0)
-    kk = orc.widen(k)
-    for (t, h), (j, g) in needles.items():
-        s = (kk[:P + t + 1, g] @ qf[t, h])
-        gap = s[j] - np.max(np.delete(s, j))
-        if gap < 30:          # another query's needle happens to align; skip that rare row
-            continue
-        assert abs(o[t, h, 0] - (j % 64)) < 1e-9 and abs(o[t, h, 1] - (100 + g)) < 1e-9
+    pool.append(pages, 0, bits(kf), bits(v))
+    o, lse = orc.attn_extend(pool, bits(qf), Hq, [0, E], synth.block_table([pages]), [P], [E], 1.0)
+    checked = 0
+    for (t, h), j in target.items():
+        assert abs(o[t, h, 0] - j) < 1e-9 and abs(o[t, h, 1] - (100 + h // G)) < 1e-9, (t, h, j)
+        assert abs(lse[t, h] - 128.0) < 1e-9
+        checked += 1
+    assert checked == E * Hq
 
 
 # ------------------------------------------------------ the paper's invariant
