@@ -24,6 +24,8 @@
 // The two query tiles ping-pong: while one tile's softmax runs, the tensor core works on the other.
 // All waits are bounded; on expiry the CTA records KV_ERR_TIMEOUT, drains its copies, frees its
 // tensor memory and returns.
+#include <type_traits>
+
 #include <cuda.h>  // CUtensorMap and its enums (types only: the encoder is looked up at run time)
 
 #include "append.cuh"
@@ -381,6 +383,7 @@ __device__ __forceinline__ void child_next(const TcArgs& a, const Item& it, Chil
 __device__ __forceinline__ int child_pages(const ChildCur& k) { return min(8, (k.len - k.jc * 128 + 15) >> 4); }
 
 // Item k of the global list: entry k / Hkv of the plan, KV head k % Hkv.  Returns false past the end.
+template <bool FAN>
 __device__ __forceinline__ bool fetch_item(const TcArgs& a, int k, int n_total, Item& it) {
   if (k >= n_total) return false;
   const int Hkv = a.pool.n_kv_heads;
@@ -389,7 +392,7 @@ __device__ __forceinline__ bool fetch_item(const TcArgs& a, int k, int n_total, 
   it.seq = r0.x; it.tp = r0.y; it.P = r0.z; it.E = r0.w;
   it.row0 = r1.x; it.n_kv[0] = r1.y; it.n_kv[1] = r1.z; it.kv_end = r1.w;
   it.c_first = 0;
-  if (a.mode == 2) {
+  if (FAN) {
     it.c_first = r1.w;
     it.kv_end = it.P;
   }
@@ -428,7 +431,8 @@ __device__ __forceinline__ void issue_pv_mmas(uint32_t o_tmem, uint32_t p_tmem, 
 
 // OPT: the softmax warps skip the search for the row maximum after an item's first tile (see there); chosen by the
 // host for batches whose sequences are long, where nearly every step is such a step.
-template <int D, bool OPT>
+// FAN: the fan-out mode (TcArgs::mode 2); the other modes are compiled without the walk over the children's tiles.
+template <int D, bool OPT, bool FAN>
 __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcArgs a, const __grid_constant__ CUtensorMap q_map) {
   using Cfg = TcCfg<D>;
   extern __shared__ unsigned char smem_raw[];
@@ -518,17 +522,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       nxt_idx = __shfl_sync(0xffffffffu, nxt_idx, 0);
       announce(round + 1, nxt_idx);
       Item it;
-      fetch_item(a, cur, n_total, it);
+      fetch_item<FAN>(a, cur, n_total, it);
       cur = nxt_idx;
       if (!ok) break;
       const int* bt = a.block_tables + (int64_t)it.seq * a.max_pages;
       const size_t head_off = (size_t)it.kvh * Cfg::kBlockBytes;
-      const int n_own = a.mode == 2 ? (it.P + 127) >> 7 : it.ld_tiles;  // tiles from the sequence's (parent's) own pages
+      const int n_own = FAN ? (it.P + 127) >> 7 : it.ld_tiles;  // tiles from the sequence's (parent's) own pages
       ChildCur cc{0, 0, 0, 0};
       for (int j = 0; j < it.ld_tiles && ok; ++j) {
         int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
         const int* src_bt = bt + j * 8;
-        if (j >= n_own) {  // fan-out mode: a tile of a child's own keys
+        if (FAN && j >= n_own) {  // fan-out mode: a tile of a child's own keys
           if (j == n_own) child_first(a, it, cc); else child_next(a, it, cc);
           np = child_pages(cc);
           src_bt = a.fan.tables + (int64_t)cc.c * a.fan.max_pages + cc.jc * 8;
@@ -588,10 +592,10 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
     uint32_t items_done[2] = {0, 0};    // items per tile so far (phase of q_full)
     bool ok = true;
     Item nxt;
-    bool has_nxt = fetch_item(a, sched_get(0), n_total, nxt);
+    bool has_nxt = fetch_item<FAN>(a, sched_get(0), n_total, nxt);
     for (int round = 0; ok && has_nxt; ++round) {
       const Item it = nxt;
-      has_nxt = fetch_item(a, sched_get(round + 1), n_total, nxt);
+      has_nxt = fetch_item<FAN>(a, sched_get(round + 1), n_total, nxt);
       sched_release(round);
       if (it.ld_tiles == 0) continue;
       {
@@ -619,11 +623,11 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         }
         if (ok && elect_one_sync()) mma_commit(smem_u32(&sm.kv_empty[stage]));
         __syncwarp();
-        const int n_own = a.mode == 2 ? (it.P + 127) >> 7 : it.ld_tiles;
+        const int n_own = FAN ? (it.P + 127) >> 7 : it.ld_tiles;
         ChildCur cc{0, 0, 0, 0};
         for (int j = 0; j < it.ld_tiles && ok; ++j) {
           int np = min(8, (it.kv_end - j * 128 + 15) >> 4);
-          if (j >= n_own) {  // fan-out mode: a tile of a child's own keys
+          if (FAN && j >= n_own) {  // fan-out mode: a tile of a child's own keys
             if (j == n_own) child_first(a, it, cc); else child_next(a, it, cc);
             np = child_pages(cc);
           }
@@ -699,7 +703,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
     uint32_t fills[2] = {0, 0};  // tiles loaded so far per buffer (phase of q_empty)
     bool ok = true;
     Item it;
-    for (int round = 0; ok && fetch_item(a, sched_get(round), n_total, it); ++round) {
+    for (int round = 0; ok && fetch_item<FAN>(a, sched_get(round), n_total, it); ++round) {
       sched_release(round);
       if (it.ld_tiles == 0) continue;
 #pragma unroll
@@ -722,7 +726,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       }
       // the next item's query tiles are asked into L2 now, a whole item ahead of their copy to shared memory
       Item nx;
-      if (fetch_item(a, sched_get(round + 1), n_total, nx) && nx.ld_tiles > 0 && lane == 0) {
+      if (fetch_item<FAN>(a, sched_get(round + 1), n_total, nx) && nx.ld_tiles > 0 && lane == 0) {
 #pragma unroll
         for (int t = 0; t < 2; ++t) {
           if (nx.n_kv[t] == 0) continue;
@@ -745,7 +749,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
     uint32_t done[2] = {0, 0};  // items finished per tile (phase of o_full / l_full, parity of inv_l)
     bool ok = true;
     Item it;
-    for (int round = 0; ok && fetch_item(a, sched_get(round), n_total, it); ++round) {
+    for (int round = 0; ok && fetch_item<FAN>(a, sched_get(round), n_total, it); ++round) {
       sched_release(round);
       if (it.ld_tiles == 0) continue;
 #pragma unroll
@@ -840,7 +844,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
       ChildCur cc{0, 0, 0, 0};
       {
         Item it;
-        const bool more_items = fetch_item(a, sched_get(round), n_total, it);
+        const bool more_items = fetch_item<FAN>(a, sched_get(round), n_total, it);
         if (!more_items) break;
         sched_release(round);
         if (it.ld_tiles == 0) continue;
@@ -851,8 +855,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         valid = tok < it.E;
         limit = valid && a.mode == 0 ? it.P + tok + 1 : it.kv_end;  // keys this row sees (rows past the end: any)
         orow_idx = (int64_t)(it.row0 + tok) * Hq + it.kvh * G + (rg & (G - 1));  // row of the LSE
-        n_own = a.mode == 2 ? (it.P + 127) >> 7 : n_t;
-        if (a.mode == 2) {
+        n_own = FAN ? (it.P + 127) >> 7 : n_t;
+        if (FAN) {
           tok_s = valid ? tok : -1;
           f_row0 = it.row0;
           cc.c = it.c_first;
@@ -871,7 +875,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) attn_extend_tc_kernel(const TcA
         // vis: how many of the tile's 128 key columns this row sees (diagonal / last tile: keys past the row's
         // limit are hidden; fan-out mode: only the row's own child, up to the row's own token)
         int vis = limit - j * 128;
-        if (j >= n_own) {
+        if (FAN && j >= n_own) {
           if (j == n_own) {
             cc.jc = 0;
             child_load(a, f_row0, cc);
@@ -1102,13 +1106,13 @@ static kv_status_t tc_grid(const kv_pool_t* p, int n_items_bound, int cta_cap, i
   return KV_OK;
 }
 
-template <int D, bool OPT>
+template <int D, bool OPT, bool FAN>
 static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid, int device, bool early_start, cudaStream_t st) {
   const size_t smem = sizeof(TcSmem<D>);
   static std::atomic<bool> configured[kMaxDevices];  // the attribute belongs to the function on one device
   if (device < 0 || device >= kMaxDevices) return KV_ERR_INVALID;
   if (!configured[device].load(std::memory_order_acquire)) {
-    KV_CUDA_OK(cudaFuncSetAttribute(attn_extend_tc_kernel<D, OPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    KV_CUDA_OK(cudaFuncSetAttribute(attn_extend_tc_kernel<D, OPT, FAN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     configured[device].store(true, std::memory_order_release);
   }
   // early_start: launched so that it may start while the plan kernel in front of it still runs (it waits for it
@@ -1124,7 +1128,7 @@ static kv_status_t launch_tc(const TcArgs& a, const CUtensorMap& q_map, int grid
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = early_start ? 1 : 0;
-  KV_CUDA_OK(cudaLaunchKernelEx(&cfg, attn_extend_tc_kernel<D, OPT>, a, q_map));
+  KV_CUDA_OK(cudaLaunchKernelEx(&cfg, attn_extend_tc_kernel<D, OPT, FAN>, a, q_map));
   count_launch();
   return KV_OK;
 }
@@ -1210,9 +1214,18 @@ kv_status_t launch_extend_tc(kv_pool_t* p, const void* q, int n_q_heads, const i
   // long-document shapes, -1 % on the 8B extend batch whose items have a dozen steps)
   const bool opt = max_total_len >= kOptimisticMinLen;
   const bool early = cta_cap >= 0;
-  if (p->head_dim == 128)
-    return opt ? launch_tc<128, true>(a, q_map, grid, p->device, early, st) : launch_tc<128, false>(a, q_map, grid, p->device, early, st);
-  return opt ? launch_tc<64, true>(a, q_map, grid, p->device, early, st) : launch_tc<64, false>(a, q_map, grid, p->device, early, st);
+  auto go = [&](auto d, auto o, auto f) {
+    return launch_tc<decltype(d)::value, decltype(o)::value, decltype(f)::value>(a, q_map, grid, p->device, early, st);
+  };
+  using I128 = std::integral_constant<int, 128>;
+  using I64 = std::integral_constant<int, 64>;
+  const bool fan_mode = mode == 2;
+  if (p->head_dim == 128) {
+    if (fan_mode) return opt ? go(I128{}, std::true_type{}, std::true_type{}) : go(I128{}, std::false_type{}, std::true_type{});
+    return opt ? go(I128{}, std::true_type{}, std::false_type{}) : go(I128{}, std::false_type{}, std::false_type{});
+  }
+  if (fan_mode) return opt ? go(I64{}, std::true_type{}, std::true_type{}) : go(I64{}, std::false_type{}, std::true_type{});
+  return opt ? go(I64{}, std::true_type{}, std::false_type{}) : go(I64{}, std::false_type{}, std::false_type{});
 }
 
 }  // namespace kvattn
