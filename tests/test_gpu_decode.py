@@ -9,6 +9,14 @@ from harness import Batch, DualPool, assert_close, run_decode, run_extend
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=[1, 2], ids=["pages-through-registers", "pages-through-shared-memory-ring"], autouse=True)
+def decode_variant(request):
+    """Every test of this file runs with both ways the decode kernel brings pages on chip."""
+    kvattn.kvattn_set_decode_impl(request.param)
+    yield request.param
+    kvattn.kvattn_set_decode_impl(0)
+
+
 @pytest.mark.parametrize("hq,hkv,d", [(4, 2, 64), (8, 8, 64), (8, 1, 64), (32, 8, 128), (8, 2, 128), (4, 4, 128)])
 def test_decode_edge_lengths(hq, hkv, d):
     geom = synth.Geometry(hq, hkv, d)
@@ -97,4 +105,20 @@ def test_decode_needle_and_position_coded_values():
             o = res["o"][i, g * geom.group]
             assert abs(o[0] - (j % 16) / 16) < 0.02 and abs(o[1] - (j // 16 % 16) / 16) < 0.02
             assert abs(o[2] - (j // 256) / 16) < 0.02
+    dp.close()
+
+
+def test_the_two_decode_variants_give_the_same_bits():
+    geom = synth.Geometry(32, 8, 128)
+    lens = [4096, 1, 16, 17, 1025, 2049, 3, 700, 0, 48]
+    dp = DualPool(geom, 1024, seed=17)
+    b = Batch(dp, [max(x, 1) for x in lens])
+    b.write([(i, 0, L) for i, L in enumerate(lens) if L > 0])
+    outs = []
+    for impl in (1, 2):
+        kvattn.kvattn_set_decode_impl(impl)
+        outs.append(run_decode(dp, b, lens, oracle=(impl == 1)))
+    assert_close(outs[0], "register variant")
+    assert np.array_equal(outs[0]["o_bits"], outs[1]["o_bits"]) and np.array_equal(outs[0]["lse_raw"], outs[1]["lse_raw"])
+    assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
     dp.close()
