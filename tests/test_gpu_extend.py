@@ -241,19 +241,21 @@ def test_more_sequences_than_the_plan_ranks():
 
 
 @pytest.mark.parametrize("impl", IMPLS)
-@pytest.mark.parametrize("hq,hkv,d", [(32, 8, 128), (4, 2, 64)])
+@pytest.mark.parametrize("hq,hkv,d", [(32, 8, 128), (4, 2, 64), (8, 1, 128)])
 def test_append_and_extend_in_one_call_is_bit_identical_to_the_two_calls(impl, hq, hkv, d):
     # attn_extend_append = kv_append(suffix) + attn_extend with fewer launches: the whole pool image, O and LSE must
     # come out bit for bit as from the two calls, and O / LSE within tolerance of the oracle.
     geom = synth.Geometry(hq, hkv, d)
     _skip_if_no_tc(impl, geom)
-    P = [0, 17, 160, 500, 31, 16, 1000]
-    E = [40, 1, 129, 64, 300, 16, 7]
+    # prefixes that end anywhere inside a page and inside a group of eight slots, suffixes of one token, of exactly a
+    # group or a page, empty ones, and ones that span several KV tiles
+    P = [0, 17, 160, 500, 31, 16, 1000, 5, 123, 8, 64, 127, 250]
+    E = [40, 1, 129, 64, 300, 16, 7, 0, 9, 8, 1, 2, 270]
     L = [p + e for p, e in zip(P, E)]
     imgs, outs = [], []
     for fused in (False, True):
-        dp = DualPool(geom, 160, seed=321)
-        b = Batch(dp, L)
+        dp = DualPool(geom, 256, seed=321)
+        b = Batch(dp, [max(x, 1) for x in L])
         b.write([(i, 0, P[i]) for i in range(len(P))])                       # the upstream operator's prefix only
         ks, vs = zip(*[b.kv(i, P[i], L[i]) for i in range(len(P))])
         if not fused:
