@@ -35,11 +35,31 @@ __device__ __forceinline__ void append_tokens(const PoolView& pool, const Append
   const int lane = threadIdx.x & 31;
   const int warps = n_warps;
   for (int token = warp_index; token < total_new; token += warps) {
-    // segment of this token: last s with cu_new[s] <= token
-    int lo = 0, hi = n_segments;
-    while (hi - lo > 1) {
-      const int mid = (lo + hi) >> 1;
-      if (__ldg(cu_new + mid) <= token) lo = mid; else hi = mid;
+    // The token's first chunks are asked for before anything else: where they go is found meanwhile (the loads do not
+    // depend on it, and a token's warp otherwise spends its time on a chain of small dependent loads).
+    const uint4* ksrc = k_new + (int64_t)token * chunks_per_token;
+    const uint4* vsrc = v_new + (int64_t)token * chunks_per_token;
+    uint4 kk[kMaxPerLane], vv[kMaxPerLane];
+#pragma unroll
+    for (int i = 0; i < kMaxPerLane; ++i) {
+      const int c = i * 32 + lane;
+      if (c < chunks_per_token) {
+        kk[i] = __ldg(ksrc + c);
+        vv[i] = __ldg(vsrc + c);
+      }
+    }
+    // segment of this token: last s with cu_new[s] <= token.  The lanes probe 32 evenly spaced entries at a time, so
+    // the search is one dependent load per factor of 32 in the number of segments instead of one per factor of 2
+    // (the chain of dependent loads is what a token's warp spends its time on).
+    int lo = 0, span = n_segments;
+    while (span > 1) {
+      const int step = (span + 31) >> 5;
+      const int idx = lo + lane * step;
+      const bool le = idx < lo + span && __ldg(cu_new + idx) <= token;
+      const int k = __popc(__ballot_sync(0xffffffffu, le)) - 1;   // >= 0: cu_new[lo] <= token
+      const int end = lo + span;
+      lo += max(k, 0) * step;
+      span = min(step, end - lo);
     }
     const int seg = lo;
     const int seg_begin = __ldg(cu_new + seg), seg_end = __ldg(cu_new + seg + 1);
@@ -51,17 +71,16 @@ __device__ __forceinline__ void append_tokens(const PoolView& pool, const Append
     const int page = __ldg(block_tables + (int64_t)row * max_pages + blk_idx);
     if (page < 0 || page >= pool.num_pages) { report(pool.status, KV_ERR_BOUNDS); continue; }
     const size_t page_off = (size_t)page * pool.n_kv_heads * blk;
-    const uint4* ksrc = k_new + (int64_t)token * chunks_per_token;
-    const uint4* vsrc = v_new + (int64_t)token * chunks_per_token;
     const bool last = token + 1 == seg_end;
     for (int c0 = 0; c0 < chunks_per_token; c0 += 32 * kMaxPerLane) {
-      uint4 kk[kMaxPerLane], vv[kMaxPerLane];
+      if (c0 > 0) {  // (the first pass's chunks are in flight already)
 #pragma unroll
-      for (int i = 0; i < kMaxPerLane; ++i) {
-        const int c = c0 + i * 32 + lane;
-        if (c < chunks_per_token) {
-          kk[i] = __ldg(ksrc + c);
-          vv[i] = __ldg(vsrc + c);
+        for (int i = 0; i < kMaxPerLane; ++i) {
+          const int c = c0 + i * 32 + lane;
+          if (c < chunks_per_token) {
+            kk[i] = __ldg(ksrc + c);
+            vv[i] = __ldg(vsrc + c);
+          }
         }
       }
 #pragma unroll
