@@ -153,6 +153,8 @@ __device__ __forceinline__ void load_page_smem(PageRegs<D>& pr, uint32_t slot, i
 
 template <int D, bool EXTEND, bool DIRECT, bool RING = false>
 __global__ void __launch_bounds__(RING ? kRingWarps * 32 : 256, 1) attn_small_kernel(SmallArgs a, int64_t total_items) {
+  // the kernel queued behind this one (the combine) may be launched while this one runs; it waits for it inside
+  ptx::launch_dependents();
   constexpr int kWarps = RING ? kRingWarps : 8;
   constexpr int kBatchPages = RING ? 2 * kChunkPages : kChunkPages;  // block-table entries held per lane pair / lane
   extern __shared__ __align__(1024) unsigned char ring_raw[];
@@ -453,6 +455,7 @@ __global__ void __launch_bounds__(256) combine_kernel(const float* __restrict__ 
                                                       int max_chunks, int chunk_tokens,
                                                       __nv_bfloat16* __restrict__ out, float* __restrict__ lse) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  ptx::dependency_wait();  // launched early: the partial results of the kernel in front are complete from here on
   if (warp >= n_rows * n_q_heads) return;
   const int row = warp / n_q_heads;
   const int len = __ldg(lens + row);
@@ -574,8 +577,19 @@ static kv_status_t launch_decode_d(kv_pool_t* p, const SmallArgs& base, int batc
     const kv_status_t ks = launch_decode_kernel<D, false>(p, a, items, ring, beside, st);
     if (ks != KV_OK) return ks;
     const int rows = batch * a.n_q_heads;
-    combine_kernel<D><<<(rows + 7) / 8, 256, 0, st>>>(a.part_o, a.part_lse, a.len_a, batch, a.n_q_heads, a.max_chunks,
-                                                      a.chunk_tokens, a.out, a.lse);
+    {
+      cudaLaunchConfig_t cfg{};
+      cfg.gridDim = dim3((unsigned)((rows + 7) / 8));
+      cfg.blockDim = dim3(256);
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      KV_CUDA_OK(cudaLaunchKernelEx(&cfg, combine_kernel<D>, (const float*)a.part_o, (const float*)a.part_lse, a.len_a, batch,
+                                    a.n_q_heads, a.max_chunks, a.chunk_tokens, a.out, a.lse));
+    }
     count_launch(2);
   }
   KV_CUDA_OK(cudaGetLastError());
