@@ -240,12 +240,16 @@ def run_ours(args):
     # the dominant kernel on its own: one launch of the attention kernel over the pages as the step left them, through
     # attn_extend_planned (the work list is built once, outside the timed region, as for the layers after the first)
     wl.extend_plan()
-    ker_ms, _ = time_steps(lambda _: wl.extend_planned(), args.steps, args.warmup, flush, world)
+    # (at most 30 launches: the denominator is the burst figure of the matmul peak, i.e. of a kernel timed alone; a
+    # long back-to-back run of this kernel settles at the power cap like the sustained matmul figure does)
+    kernel_steps = min(args.steps, 30)
+    ker_ms, _ = time_steps(lambda _: wl.extend_planned(), kernel_steps, args.warmup, flush, world)
     ext_kernel_ms = statistics.mean(ker_ms)
     ext_tflops = flops / (ext_kernel_ms * 1e-3) / 1e12
-    call_ms, _ = time_steps(lambda _: wl.extend(), args.steps, args.warmup, flush, world)   # attn_extend: plan + kernel
+    side_steps = min(args.steps, 20)   # the two comparison figures need no long runs
+    call_ms, _ = time_steps(lambda _: wl.extend(), side_steps, args.warmup, flush, world)   # attn_extend: plan + kernel
     # the same step as two calls (kv_append, then attn_extend), for comparison
-    two_ms, _ = time_steps(lambda _: (wl.append_suffix(), wl.extend()), args.steps, args.warmup, flush, world)
+    two_ms, _ = time_steps(lambda _: (wl.append_suffix(), wl.extend()), min(args.steps, 20), args.warmup, flush, world)
 
     # ---- e2e: host buffers, copies inside the timed region ---------------------------------
     e = wl.ext
@@ -315,7 +319,7 @@ def run_ours(args):
         "roofline": {"bound": "tensor", "kernel": "attn_extend_tc_kernel (attn_extend_planned)", "achieved": round(ext_tflops, 3),
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(ext_tflops / peaks["bf16_tflops"], 4),
                      "peak_source": f"{peaks['source']} (burst bf16 matmul)", "frac_of_nominal_2250": round(ext_tflops / 2250.0, 4),
-                     "kernel_ms": round(ext_kernel_ms, 5), "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                     "kernel_ms": round(ext_kernel_ms, 5), "kernel_launches_timed": kernel_steps, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
                      "target_frac_of_dense_bf16_peak": 0.60,
                      "target_met_vs_measured_peak": bool(ext_tflops / peaks["bf16_tflops"] >= 0.60),
                      "target_met_vs_nominal_2250": bool(ext_tflops / 2250.0 >= 0.60)},
