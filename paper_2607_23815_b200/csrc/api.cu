@@ -312,7 +312,9 @@ kv_status_t attn_mixed(kv_pool_t* p, int n_q_heads, float scale, const attn_exte
                        const attn_decode_args_t* dec, void* workspace, size_t workspace_bytes, void* stream) {
   if (p == nullptr || !on_pool_device(p)) return KV_ERR_INVALID;
   if (!heads_supported(p, n_q_heads)) return KV_ERR_UNSUPPORTED;
-  const bool has_ext = ext != nullptr && ext->batch > 0 && ext->total_q > 0;
+  // (an extend set that launches nothing must not count: the decode kernel may only be queued to start early behind a
+  // kernel of this call, never behind whatever the caller ran before)
+  const bool has_ext = ext != nullptr && ext->batch > 0 && ext->total_q > 0 && ext->max_extend_len > 0;
   const bool has_dec = dec != nullptr && dec->batch > 0;
   cudaStream_t st = (cudaStream_t)stream;
   size_t ext_bytes = 0;
