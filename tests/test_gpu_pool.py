@@ -104,6 +104,35 @@ def test_append_is_bit_exact_over_the_whole_pool_image(geom):
     dp.close()
 
 
+@pytest.mark.parametrize("n_seq", [1, 31, 33, 1025, 3000])
+def test_append_with_many_and_empty_segments_is_bit_exact(n_seq):
+    # The segment of a token is found by a search over cu_new in which the lanes probe 32 entries per step: segment
+    # counts around the powers of 32, runs of empty segments (equal entries of cu_new) and one-token segments.
+    geom = synth.Geometry(2, 1, 64)
+    rng = np.random.default_rng(n_seq)
+    lens = [int(x) for x in rng.choice([0, 0, 1, 2, 5, 16, 17], size=n_seq)]
+    if sum(lens) == 0:
+        lens[-1] = 3
+    pages = sum(synth.pages_needed(max(L, 1), 16) for L in lens) + 4
+    dp = DualPool(geom, pages, seed=600 + n_seq)
+    b = Batch(dp, [max(L, 1) for L in lens])
+    ks, vs = zip(*[b.kv(i, 0, lens[i]) for i in range(n_seq)])
+    dp.append(b.rows, [(i, 0) for i in range(n_seq)], list(ks), list(vs))          # one call, n_seq segments
+    torch.cuda.synchronize()
+    assert kvattn.kv_last_async_status(dp.pool) == kvattn.KV_OK
+    k_img, v_img = dp.device_image()
+    for i, L in enumerate(lens):
+        if L == 0:
+            assert np.all(k_img[b.rows[i]] == NAN_BITS)                            # an empty segment writes nothing
+            continue
+        gk, gv = dp.host.gather(b.rows[i], L)
+        dk = np.concatenate([k_img[pg].transpose(1, 0, 2) for pg in b.rows[i]])
+        dv = np.concatenate([v_img[pg].transpose(1, 0, 2) for pg in b.rows[i]])
+        assert np.array_equal(dk[:L], gk) and np.array_equal(dv[:L], gv), i
+        assert np.all(dk[L:] == 0) and np.all(dv[L:] == 0), i
+    dp.close()
+
+
 @pytest.mark.parametrize("geom", GEOMS, ids=["d64", "d128"])
 def test_gather_returns_what_was_appended(geom):
     dp = DualPool(geom, 32, seed=12)
