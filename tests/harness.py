@@ -33,7 +33,7 @@ class DualPool:
     def __init__(self, geom: synth.Geometry, num_pages: int, seed: int, device="cuda", fill=NAN_BITS,
                  with_oracle=True):
         self.geom, self.num_pages, self.seed, self.device = geom, num_pages, seed, device
-        self.gen_device = device        # where the input generator runs ("cpu": no generator kernels on the GPU)
+        self.gen_device = "cpu"         # the input generator runs on the host, so that nearly every kernel a test launches is the library's
         n_elem = num_pages * geom.n_kv_heads * geom.page_size * geom.head_dim
         # caller-owned buffers, pre-filled (NaN by default) so that any stale read shows up
         self.k_buf = torch.full((n_elem,), fill, dtype=torch.int16, device=device)
