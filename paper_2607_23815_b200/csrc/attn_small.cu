@@ -256,6 +256,7 @@ __global__ void __launch_bounds__(RING ? kRingWarps * 32 : 256, 1) attn_small_ke
   const int first_page = chunk_begin >> 4;
   const int n_pages = (chunk_end - chunk_begin + 15) >> 4;
 
+  const uint64_t ring_policy = RING ? ptx::l2_evict_first_policy() : 0;
   uint32_t ring_issued = 0, ring_used = 0;  // ring variant: pages asked for / consumed so far (slot and phase follow)
   for (int pb = 0; pb < n_pages; pb += kBatchPages) {
     const int np = min(kBatchPages, n_pages - pb);
@@ -359,8 +360,10 @@ __global__ void __launch_bounds__(RING ? kRingWarps * 32 : 256, 1) attn_small_ke
           const uint32_t s = ring_issued % kRingStages;
           const uint32_t slot = slots + s * (2 * 16 * D * 2), bar = bars + s * 8;
           ptx::mbar_arrive_expect_tx(bar, 2 * 16 * D * 2);
-          ptx::bulk_g2s(slot, kbase + (size_t)pg * page_stride, 16 * D * 2, bar);
-          ptx::bulk_g2s(slot + 16 * D * 2, vbase + (size_t)pg * page_stride, 16 * D * 2, bar);
+          // (every page is read once: its lines are the first to leave L2, not the K/V that the extend kernel beside
+          // this one re-reads)
+          ptx::bulk_g2s_hint(slot, kbase + (size_t)pg * page_stride, 16 * D * 2, bar, ring_policy);
+          ptx::bulk_g2s_hint(slot + 16 * D * 2, vbase + (size_t)pg * page_stride, 16 * D * 2, bar, ring_policy);
         }
         ++ring_issued;
       };
