@@ -313,9 +313,9 @@ kv_status_t kvattn_set_extend_impl(int impl);
 /* Test/tuning hook for attn_extend_shared: 0 = choose by the mean suffix length (default), 1 = three kernels
  * (shared part, own part, merge), 2 = one kernel that walks the parent's and then the children's tiles. */
 kv_status_t kvattn_set_shared_impl(int impl);
-/* Selects how the decode kernel brings pages on chip: 0 = default, 1 = straight into registers (one page per warp in
- * flight), 2 = through a per-warp ring of page slots in shared memory filled by bulk copies (several pages per warp in
- * flight).  Same arithmetic, same bits.  Process-wide; for tests and benchmarks. */
+/* Selects how the decode kernel brings pages on chip: 1 = straight into registers (one page per warp in flight), 2 =
+ * through a per-warp ring of page slots in shared memory filled by bulk copies (several pages per warp in flight);
+ * 0 = the default, which is 2.  Same arithmetic, same bits.  Process-wide; for tests and benchmarks. */
 kv_status_t kvattn_set_decode_impl(int impl);
 /* Tuning: inside attn_mixed (both sets present) the persistent extend kernel takes at most n SMs, so that the
  * HBM-bound decode kernel runs beside it on the others instead of after it.  0 = derived from the bounds of the two

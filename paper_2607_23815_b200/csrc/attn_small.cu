@@ -506,7 +506,7 @@ size_t decode_workspace_bytes(int n_q_heads, int head_dim, int batch, int max_ct
   return align256(slots * head_dim * sizeof(float)) + align256(slots * sizeof(float));
 }
 
-std::atomic<int> g_decode_impl{0};  // 0: default, 1: pages stream through registers, 2: pages go through a shared-memory ring
+std::atomic<int> g_decode_impl{0};  // 0: default (the ring), 1: pages stream through registers, 2: pages go through a shared-memory ring
 
 // Launches the partial (or direct) decode kernel in the chosen variant.
 template <int D, bool DIRECT>
@@ -544,10 +544,10 @@ template <int D>
 static kv_status_t launch_decode_d(kv_pool_t* p, const SmallArgs& base, int batch, int max_ctx_len, void* workspace,
                                    size_t workspace_bytes, bool beside, cudaStream_t st) {
   SmallArgs a = base;
-  // beside the tensor-core kernel the ring variant is the default: it keeps more bytes in flight per SM, so the SMs the
-  // other kernel leaves free come closer to the memory's bandwidth (measured: mixed step 0.46 -> 0.42 ms)
-  const int impl = g_decode_impl.load();
-  const bool ring = impl == 2 || (impl == 0 && beside);
+  // The ring variant is the default: it keeps more bytes in flight per SM, which holds the bandwidth up on the SMs the
+  // tensor-core kernel leaves free in a mixed step (0.46 -> 0.42 ms) and, alone, is worth 1.5 % on long contexts
+  // (6190 vs 6100 GB/s on 256 sequences of 1024-4096 tokens) and nothing either way on shorter ones.
+  const bool ring = g_decode_impl.load() != 1;
   a.max_row_tiles = 1;
   a.chunk_tokens = kDecodeChunkTokens;
   a.max_chunks = (max_ctx_len + kDecodeChunkTokens - 1) / kDecodeChunkTokens;
