@@ -37,7 +37,7 @@ HEADLINE = "extend_8b"
 
 # DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum) from the
 # ncu captures summarised under profiles/; None until a capture of that kernel/workload exists.
-NCU_TRAFFIC_BYTES = {"extend_8b": 603_000_000, "decode_8b": 2_651_000_000}  # profiles/attn_*_kernel_*.md
+NCU_TRAFFIC_BYTES = {"extend_8b": 603_000_000, "decode_8b": 2_652_000_000}  # profiles/attn_*_kernel_*.md
 
 
 def load_peaks():
