@@ -228,6 +228,20 @@ def run_ours(args):
         # of the headline step alone lasts a few milliseconds, too short for more than a handful of samples
         box["sampler"] = ClockSampler(dev.index or 0)
 
+    # ---- the dominant kernel on its own, BEFORE the long step loop: one launch of the attention kernel over the pages
+    # as a step leaves them, through attn_extend_planned (the work list is built once, outside the timed region, as for
+    # the layers after the first).  At most 30 launches, and in front of the step loop rather than behind it: the
+    # denominator is the burst figure of the matmul peak, i.e. of a kernel timed alone on a GPU that has not been at
+    # its power cap for tens of milliseconds; back-to-back launches of this kernel behind a 100-step loop settle 3 %
+    # lower, like the sustained matmul figure does (inside a step, where the prologue kernel gives the tensor cores a
+    # pause, the kernel takes step minus prologue = the time measured here).
+    for _ in range(3):
+        wl.extend_append()
+    wl.extend_plan()
+    kernel_steps = min(args.steps, 30)
+    ker_ms, _ = time_steps(lambda _: wl.extend_planned(), kernel_steps, args.warmup, flush, world)
+    ext_kernel_ms = statistics.mean(ker_ms)
+
     def timed_start():
         box["l0"] = kvattn.kvattn_launch_count()
 
@@ -237,14 +251,6 @@ def run_ours(args):
     flops = wl.ext.flops(g)
     all_flops = sum_over_ranks(flops, world)
     value = all_flops / (ms_step * 1e-3) / 1e12
-    # the dominant kernel on its own: one launch of the attention kernel over the pages as the step left them, through
-    # attn_extend_planned (the work list is built once, outside the timed region, as for the layers after the first)
-    wl.extend_plan()
-    # (at most 30 launches: the denominator is the burst figure of the matmul peak, i.e. of a kernel timed alone; a
-    # long back-to-back run of this kernel settles at the power cap like the sustained matmul figure does)
-    kernel_steps = min(args.steps, 30)
-    ker_ms, _ = time_steps(lambda _: wl.extend_planned(), kernel_steps, args.warmup, flush, world)
-    ext_kernel_ms = statistics.mean(ker_ms)
     ext_tflops = flops / (ext_kernel_ms * 1e-3) / 1e12
     side_steps = min(args.steps, 20)   # the two comparison figures need no long runs
     call_ms, _ = time_steps(lambda _: wl.extend(), side_steps, args.warmup, flush, world)   # attn_extend: plan + kernel
@@ -319,7 +325,8 @@ def run_ours(args):
         "roofline": {"bound": "tensor", "kernel": "attn_extend_tc_kernel (attn_extend_planned)", "achieved": round(ext_tflops, 3),
                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(ext_tflops / peaks["bf16_tflops"], 4),
                      "peak_source": f"{peaks['source']} (burst bf16 matmul)", "frac_of_nominal_2250": round(ext_tflops / 2250.0, 4),
-                     "kernel_ms": round(ext_kernel_ms, 5), "kernel_launches_timed": kernel_steps, "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+                     "kernel_ms": round(ext_kernel_ms, 5), "kernel_launches_timed": kernel_steps,
+                     "kernel_loop": "attn_extend_planned alone, timed in front of the step loop", "traffic": NCU_TRAFFIC_BYTES.get(w.name),
                      "target_frac_of_dense_bf16_peak": 0.60,
                      "target_met_vs_measured_peak": bool(ext_tflops / peaks["bf16_tflops"] >= 0.60),
                      "target_met_vs_nominal_2250": bool(ext_tflops / 2250.0 >= 0.60)},
