@@ -235,8 +235,6 @@ def run_ours(args):
     # its power cap for tens of milliseconds; back-to-back launches of this kernel behind a 100-step loop settle 3 %
     # lower, like the sustained matmul figure does (inside a step, where the prologue kernel gives the tensor cores a
     # pause, the kernel takes step minus prologue = the time measured here).
-    for _ in range(3):
-        wl.extend_append()
     wl.extend_plan()
     kernel_steps = min(args.steps, 30)
     ker_ms, _ = time_steps(lambda _: wl.extend_planned(), kernel_steps, args.warmup, flush, world)
